@@ -1,0 +1,210 @@
+"""CPU oracle for the active-weight hot path (test infrastructure only).
+
+A thin ctypes front for ``afx_oracle.c`` plus the decoder-layer composition in
+``oracle.layer``.  Nothing here is part of the product: only the tests, the smoke
+check and the benchmark's CPU-baseline leg may import it, and it imports nothing
+from the CUDA package.  Arrays of 16-bit floats are numpy ``uint16`` bit patterns;
+``dtype`` is ``"f16"`` or ``"bf16"``.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "afx_oracle.c")
+_SO = os.path.join(_HERE, "libafx_oracle.so")
+
+DTYPES = {"f16": 0, "bf16": 1}
+TOPK, THRESHOLD = 0, 1
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (OpenMP only spreads independent output rows)."""
+    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
+        tmp = _SO + f".{os.getpid()}.tmp"
+        subprocess.check_call(
+            ["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-o", tmp, _SRC, "-lm"]
+        )
+        os.replace(tmp, _SO)
+    return _SO
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+    return _lib
+
+
+def _p(a, ct):
+    return a.ctypes.data_as(ctypes.POINTER(ct))
+
+
+def _u16(a):
+    a = np.ascontiguousarray(a)
+    assert a.dtype == np.uint16, a.dtype
+    return a
+
+
+def threads() -> int:
+    return int(lib().afxo_threads())
+
+
+def decode(bits, dtype: str) -> np.ndarray:
+    """fp64 values of 16-bit patterns."""
+    bits = _u16(bits)
+    out = np.empty(bits.shape, np.float64)
+    lib().afxo_decode(_p(bits, ctypes.c_uint16), ctypes.c_int64(bits.size), DTYPES[dtype],
+                      _p(out, ctypes.c_double))
+    return out
+
+
+def round_to(values, dtype: str) -> np.ndarray:
+    """Round fp64 values once (nearest-even) to 16-bit patterns."""
+    v = np.ascontiguousarray(values, np.float64)
+    out = np.empty(v.shape, np.uint16)
+    lib().afxo_round(_p(v, ctypes.c_double), ctypes.c_int64(v.size), DTYPES[dtype],
+                     _p(out, ctypes.c_uint16))
+    return out
+
+
+def select_active(x, dtype: str, mode: int, k: int = 0, tau: float = 0.0) -> np.ndarray:
+    """Ascending active-channel list of x[T][K] (union over the T tokens)."""
+    x = _u16(x)
+    if x.ndim == 1:
+        x = x[None, :]
+    T, K = x.shape
+    idx = np.empty(K, np.int32)
+    cnt = ctypes.c_int32(0)
+    rc = lib().afxo_select_active(_p(x, ctypes.c_uint16), DTYPES[dtype], K, T, mode, int(k),
+                                  ctypes.c_float(tau), _p(idx, ctypes.c_int32),
+                                  ctypes.byref(cnt))
+    if rc != 0:
+        raise ValueError("afxo_select_active: bad argument")
+    return idx[: cnt.value].copy()
+
+
+def diff_active(idxA, idxP, K: int):
+    """(miss = A \\ P ascending, hit = |A & P|) for ascending lists A, P."""
+    A = np.ascontiguousarray(idxA, np.int32)
+    P = np.ascontiguousarray(idxP, np.int32)
+    miss = np.empty(max(A.size, 1), np.int32)
+    nm, nh = ctypes.c_int32(0), ctypes.c_int32(0)
+    rc = lib().afxo_diff_active(_p(A, ctypes.c_int32), A.size, _p(P, ctypes.c_int32), P.size, K,
+                                _p(miss, ctypes.c_int32), ctypes.byref(nm), ctypes.byref(nh))
+    if rc != 0:
+        raise ValueError("afxo_diff_active: bad argument")
+    return miss[: nm.value].copy(), nh.value
+
+
+def sparse_gemv(Wt, dtype: str, N: int, x, idx, slot=None) -> np.ndarray:
+    """y[T][N] (fp64) = sum_c x[t][idx[c]] * Wt[col(c)][:N]; Wt is [rows][ldw] bit patterns."""
+    Wt = _u16(Wt)
+    x = _u16(x)
+    if x.ndim == 1:
+        x = x[None, :]
+    T, K = x.shape
+    ldw = Wt.shape[1]
+    idx = np.ascontiguousarray(idx, np.int32)
+    y = np.empty((T, N), np.float64)
+    sp = None
+    if slot is not None:
+        slot = np.ascontiguousarray(slot, np.int32)
+        sp = _p(slot, ctypes.c_int32)
+    rc = lib().afxo_sparse_gemv(_p(Wt, ctypes.c_uint16), DTYPES[dtype], K, N,
+                                ctypes.c_int64(ldw), _p(x, ctypes.c_uint16), T,
+                                _p(idx, ctypes.c_int32), idx.size, sp, _p(y, ctypes.c_double))
+    if rc != 0:
+        raise ValueError("afxo_sparse_gemv: bad argument")
+    return y
+
+
+def rmsnorm(h, g, eps: float, dtype: str) -> np.ndarray:
+    h = np.ascontiguousarray(h, np.float64)
+    if h.ndim == 1:
+        h = h[None, :]
+    g = np.ascontiguousarray(g, np.float64)
+    T, H = h.shape
+    out = np.empty((T, H), np.uint16)
+    lib().afxo_rmsnorm(_p(h, ctypes.c_double), _p(g, ctypes.c_double), T, H, ctypes.c_double(eps),
+                       DTYPES[dtype], _p(out, ctypes.c_uint16))
+    return out
+
+
+def rope(v, pos, theta: float = 10000.0) -> np.ndarray:
+    """Rotate v[T][heads][D] (fp64) by the positions pos[T]; returns a new array."""
+    v = np.array(v, np.float64, order="C", copy=True)
+    T, heads, D = v.shape
+    pos = np.ascontiguousarray(pos, np.int32)
+    lib().afxo_rope(_p(v, ctypes.c_double), T, heads, D, _p(pos, ctypes.c_int32),
+                    ctypes.c_double(theta))
+    return v
+
+
+def attention(q, kc, vc, L: int, dtype: str) -> np.ndarray:
+    """q[q_heads][D] fp64, kc/vc [>=L][kv_heads][D] fp16 bits -> out[q_heads][D] dtype bits."""
+    q = np.ascontiguousarray(q, np.float64)
+    kc, vc = _u16(kc), _u16(vc)
+    q_heads, D = q.shape
+    kv_heads = kc.shape[1]
+    out = np.empty((q_heads, D), np.uint16)
+    lib().afxo_attention(_p(q, ctypes.c_double), _p(kc, ctypes.c_uint16), _p(vc, ctypes.c_uint16),
+                         L, q_heads, kv_heads, D, DTYPES[dtype], _p(out, ctypes.c_uint16))
+    return out
+
+
+def silu_mul(g, u, dtype: str) -> np.ndarray:
+    g = np.ascontiguousarray(g, np.float64)
+    u = np.ascontiguousarray(u, np.float64)
+    out = np.empty(g.shape, np.uint16)
+    lib().afxo_silu_mul(_p(g, ctypes.c_double), _p(u, ctypes.c_double), ctypes.c_int64(g.size),
+                        DTYPES[dtype], _p(out, ctypes.c_uint16))
+    return out
+
+
+class LfuCache:
+    """Context-level LFU column cache of one weight tensor (Sec. 4.2), state on the host."""
+
+    def __init__(self, K: int, capacity: int):
+        self.K, self.C = int(K), int(capacity)
+        self.slot_of = np.full(K, -1, np.int32)
+        self.chan_of = np.full(capacity, -1, np.int32)
+        self.freq = np.zeros(K, np.uint32)
+
+    def reset_counts(self):
+        """New sequence: the usage count of every channel starts from zero."""
+        self.freq[:] = 0
+
+    def install(self, channels):
+        """Pre-load channels into the lowest free slots (initial cache contents)."""
+        for j in channels:
+            s = int(np.flatnonzero(self.chan_of < 0)[0])
+            self.chan_of[s] = j
+            self.slot_of[j] = s
+
+    def step(self, idx):
+        """Returns dict(slot, fetched, hits, misses, transients) for one token's active list."""
+        idx = np.ascontiguousarray(idx, np.int32)
+        slot = np.empty(max(idx.size, 1), np.int32)
+        fetched = np.empty(max(idx.size, 1), np.int32)
+        nh, nm, nt = ctypes.c_int32(0), ctypes.c_int32(0), ctypes.c_int32(0)
+        rc = lib().afxo_cache_step(self.K, self.C, _p(self.slot_of, ctypes.c_int32),
+                                   _p(self.chan_of, ctypes.c_int32),
+                                   _p(self.freq, ctypes.c_uint32), _p(idx, ctypes.c_int32),
+                                   idx.size, _p(slot, ctypes.c_int32),
+                                   _p(fetched, ctypes.c_int32), ctypes.byref(nh),
+                                   ctypes.byref(nm), ctypes.byref(nt))
+        if rc != 0:
+            raise ValueError("afxo_cache_step: bad argument")
+        return dict(slot=slot[: idx.size].copy(), fetched=fetched[: nm.value].copy(),
+                    hits=nh.value, misses=nm.value, transients=nt.value)
+
+    def cached(self) -> np.ndarray:
+        return np.sort(self.chan_of[self.chan_of >= 0])

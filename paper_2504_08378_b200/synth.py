@@ -1,0 +1,113 @@
+"""Seeded synthetic inputs shared by the CUDA path's tests, the oracle's tests and the bench.
+
+This module only *draws inputs*: random weights, activations, caches and channel
+activity patterns with the shapes and value distributions of the Llama-shaped
+decode workloads.  It holds none of the method's arithmetic (no selection, no
+GEMV, no cache policy) and imports neither the CUDA binding nor the oracle.
+
+All 16-bit float arrays are numpy ``uint16`` bit patterns; ``dtype`` is ``"f16"``
+(IEEE binary16) or ``"bf16"``.  Streams are Philox counters keyed by
+``(seed, stream id)``, so any tensor can be regenerated on its own.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+DTYPES = ("f16", "bf16")
+
+
+def rng(seed: int, stream: int) -> np.random.Generator:
+    return np.random.Generator(np.random.Philox(key=[int(seed) & (2**64 - 1), int(stream) & (2**64 - 1)]))
+
+
+def f32_to_bits(a, dtype: str) -> np.ndarray:
+    """Round float32 values to nearest-even 16-bit patterns."""
+    a = np.ascontiguousarray(a, np.float32)
+    if dtype == "f16":
+        return a.astype(np.float16).view(np.uint16)
+    if dtype == "bf16":
+        u = a.view(np.uint32)
+        nan = np.isnan(a)
+        r = ((u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) >> np.uint32(16)).astype(np.uint16)
+        if nan.any():
+            r = np.where(nan, np.uint16(0x7FC0), r)
+        return r
+    raise ValueError(dtype)
+
+
+def bits_to_f32(bits, dtype: str) -> np.ndarray:
+    bits = np.ascontiguousarray(bits, np.uint16)
+    if dtype == "f16":
+        return bits.view(np.float16).astype(np.float32)
+    if dtype == "bf16":
+        return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32)
+    raise ValueError(dtype)
+
+
+def normal_bits(seed: int, stream: int, shape, sigma: float, dtype: str) -> np.ndarray:
+    """N(0, sigma^2) values rounded to dtype; used for weights and KV caches."""
+    g = rng(seed, stream)
+    a = g.standard_normal(size=shape, dtype=np.float32)
+    a *= np.float32(sigma)
+    return f32_to_bits(a, dtype)
+
+
+def weight(seed: int, stream: int, K: int, N: int, dtype: str, sigma: float = 0.02,
+           ldw: int | None = None) -> np.ndarray:
+    """Channel-contiguous operator weight Wt[K][ldw]; columns N..ldw are zero padding."""
+    ldw = N if ldw is None else ldw
+    w = normal_bits(seed, stream, (K, N), sigma, dtype)
+    if ldw == N:
+        return w
+    out = np.zeros((K, ldw), np.uint16)
+    out[:, :N] = w
+    return out
+
+
+def laplace(seed: int, stream: int, shape, scale: float = 1.0) -> np.ndarray:
+    """Laplace(0, scale) by inverse CDF of seeded uniforms (float64)."""
+    u = rng(seed, stream).random(size=shape) - 0.5
+    return -scale * np.sign(u) * np.log1p(-2.0 * np.abs(u))
+
+
+def laplace_bits(seed: int, stream: int, shape, dtype: str, scale: float = 1.0) -> np.ndarray:
+    return f32_to_bits(laplace(seed, stream, shape, scale).astype(np.float32), dtype)
+
+
+def laplace_tau(p: float, scale: float = 1.0) -> float:
+    """Magnitude below which a fraction p of Laplace(0, scale) draws fall (|x| ~ Exp(1/scale)).
+
+    p = 0 returns -1, the "keep every channel" setting of the threshold mode.
+    """
+    if p <= 0.0:
+        return -1.0
+    return float(-scale * np.log1p(-p))
+
+
+def keep_count(K: int, sparsity_percent: int) -> int:
+    """Channels kept at an integer sparsity percentage: K - floor(K * p / 100)."""
+    return int(K - (K * int(sparsity_percent)) // 100)
+
+
+def channel_scales(seed: int, stream: int, K: int, sigma: float = 0.5) -> np.ndarray:
+    """Persistent per-channel lognormal scale: gives successive layers similar |x| profiles."""
+    return np.exp(sigma * rng(seed, stream).standard_normal(K))
+
+
+def zipf_activity_bits(seed: int, stream: int, K: int, dtype: str, alpha: float = 1.1,
+                       perm_stream: int = 0) -> np.ndarray:
+    """One activation vector whose top-k sets follow a Zipf(alpha) channel popularity.
+
+    Channel weights w_r ~ r^-alpha are laid over a seeded permutation shared by all steps
+    of a tensor (``perm_stream``); score_j = ln w_j + Gumbel noise, so the k largest scores
+    are a weighted sample without replacement.  |x_j| = exp(score_j / 4) keeps the values
+    inside fp16/bf16 range while preserving the order; signs are random.
+    """
+    perm = rng(seed, perm_stream).permutation(K)
+    rank = np.empty(K, np.int64)
+    rank[perm] = np.arange(1, K + 1)
+    g = rng(seed, stream)
+    score = -alpha * np.log(rank.astype(np.float64)) + g.gumbel(size=K)
+    mag = np.exp(score / 4.0)
+    sign = np.where(g.random(K) < 0.5, -1.0, 1.0)
+    return f32_to_bits((mag * sign).astype(np.float32), dtype)
