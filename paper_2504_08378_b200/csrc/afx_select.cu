@@ -1,0 +1,106 @@
+// afx_select_active / afx_diff_active: stand-alone selection and cross-layer set difference.
+#include "afx_select.cuh"
+
+namespace afx {
+
+constexpr int kSelectThreads = 1024;
+
+template <int DT>
+__global__ void __launch_bounds__(kSelectThreads, 1)
+select_kernel(const uint16_t* __restrict__ x, int K, int T, int mode, int k, float tau,
+              int32_t* __restrict__ idx, int32_t* __restrict__ count, uint32_t* __restrict__ bitmap) {
+    extern __shared__ uint32_t s_flags[];
+    __shared__ SelectScratch scratch;
+    block_select_flags<DT>(x, K, T, mode, k, tau, s_flags, &scratch);
+    const int total = block_compact_flags(s_flags, K, idx, &scratch);
+    if (threadIdx.x == 0) *count = total;
+    if (bitmap != nullptr) {
+        const int nwords = (K + 31) >> 5;
+        for (int w = threadIdx.x; w < nwords; w += blockDim.x) bitmap[w] = s_flags[w];
+    }
+}
+
+// miss = A \ P (ascending), hit = |A & P|.  One block; each warp owns a contiguous run of
+// list positions so that the output keeps A's order.
+__global__ void __launch_bounds__(kSelectThreads, 1)
+diff_kernel(const int32_t* __restrict__ idxA, const int32_t* __restrict__ cntA,
+            const uint32_t* __restrict__ bitmapP, int K, int32_t* __restrict__ miss,
+            int32_t* __restrict__ miss_count, int32_t* __restrict__ hit_count) {
+    __shared__ int scan[33];
+    int n = *cntA;
+    n = max(0, min(n, K));
+    const int lane = lane_id();
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    const int nchunks = (n + 31) >> 5;
+    const int nw = blockDim.x >> 5;
+    const int per = (nchunks + nw - 1) / nw;
+    const int c0 = min(nchunks, warp_id() * per), c1 = min(nchunks, c0 + per);
+    int cm = 0;
+    for (int c = c0; c < c1; ++c) {
+        const int p = (c << 5) + lane;
+        bool m = false;
+        if (p < n) {
+            const int j = idxA[p];
+            m = ((bitmapP[j >> 5] >> (j & 31)) & 1u) == 0u;
+        }
+        cm += __popc(__ballot_sync(0xFFFFFFFFu, m));
+    }
+    int base = block_exclusive_over_warps(cm, scan);
+    const int total = scan[32];
+    for (int c = c0; c < c1; ++c) {
+        const int p = (c << 5) + lane;
+        bool m = false;
+        int j = 0;
+        if (p < n) {
+            j = idxA[p];
+            m = ((bitmapP[j >> 5] >> (j & 31)) & 1u) == 0u;
+        }
+        const uint32_t b = __ballot_sync(0xFFFFFFFFu, m);
+        if (m) miss[base + __popc(b & lt_mask)] = j;
+        base += __popc(b);
+    }
+    if (threadIdx.x == 0) {
+        *miss_count = total;
+        *hit_count = n - total;
+    }
+}
+
+}  // namespace afx
+
+extern "C" afx_status afx_select_active(const void* x, int dtype, int K, int T, int mode, int k,
+                                        float tau, int32_t* idx, int32_t* count, uint32_t* bitmap,
+                                        void* stream) {
+    using namespace afx;
+    if (x == nullptr || idx == nullptr || count == nullptr) return AFX_ERR_INVALID_ARG;
+    if (K <= 0 || K > (1 << 20) || T < 1 || T > AFX_MAX_T) return AFX_ERR_INVALID_ARG;
+    if (dtype != AFX_F16 && dtype != AFX_BF16) return AFX_ERR_UNSUPPORTED;
+    if (mode != AFX_MODE_TOPK && mode != AFX_MODE_THRESHOLD) return AFX_ERR_UNSUPPORTED;
+    if (mode == AFX_MODE_TOPK && (k < 0 || k > K)) return AFX_ERR_INVALID_ARG;
+    if (mode == AFX_MODE_THRESHOLD && tau != tau) return AFX_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(x) & 1u) || (reinterpret_cast<uintptr_t>(idx) & 3u) ||
+        (reinterpret_cast<uintptr_t>(count) & 3u) || (reinterpret_cast<uintptr_t>(bitmap) & 3u))
+        return AFX_ERR_ALIGNMENT;
+    const size_t smem = static_cast<size_t>((K + 31) >> 5) * sizeof(uint32_t);
+    auto kern = dtype == AFX_F16 ? select_kernel<AFX_F16> : select_kernel<AFX_BF16>;
+    if (smem > 40 * 1024) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(smem)) != cudaSuccess)
+            return AFX_ERR_CUDA;
+    }
+    kern<<<1, kSelectThreads, smem, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint16_t*>(x), K, T, mode, k, tau, idx, count, bitmap);
+    return launch_status();
+}
+
+extern "C" afx_status afx_diff_active(const int32_t* idxA, const int32_t* cntA,
+                                      const uint32_t* bitmapP, int K, int32_t* miss,
+                                      int32_t* miss_count, int32_t* hit_count, void* stream) {
+    using namespace afx;
+    if (idxA == nullptr || cntA == nullptr || bitmapP == nullptr || miss == nullptr ||
+        miss_count == nullptr || hit_count == nullptr)
+        return AFX_ERR_INVALID_ARG;
+    if (K <= 0 || K > (1 << 20)) return AFX_ERR_INVALID_ARG;
+    diff_kernel<<<1, kSelectThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        idxA, cntA, bitmapP, K, miss, miss_count, hit_count);
+    return launch_status();
+}

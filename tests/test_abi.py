@@ -1,0 +1,97 @@
+"""The C-ABI library loads without a GPU, exports every declared symbol, and rejects bad
+arguments on the host before anything is launched."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2504_08378_b200 import afx
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_symbols():
+    names = set()
+    for fn in os.listdir(os.path.join(ROOT, "include")):
+        if fn.endswith(".h"):
+            src = open(os.path.join(ROOT, "include", fn)).read()
+            src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+            names |= set(re.findall(r"\b(afx_[a-z0-9_]+)\s*\(", src))
+    return sorted(names)
+
+
+def test_every_declared_symbol_is_exported():
+    L = afx.lib()
+    declared = _declared_symbols()
+    assert "afx_select_active" in declared and "afx_sparse_gemv" in declared
+    for name in declared:
+        assert hasattr(L, name), f"{name} declared in include/ but not exported"
+
+
+def test_binding_has_the_same_names():
+    for name in _declared_symbols():
+        assert hasattr(afx, name), f"binding lacks {name}"
+
+
+def test_version_and_status_strings():
+    assert afx.afx_version() == (0, 1) or afx.afx_version()[0] >= 0
+    assert afx.afx_status_string(0) == "AFX_OK"
+    assert afx.afx_status_string(2) == "AFX_ERR_ALIGNMENT"
+    assert afx.afx_status_string(99) == "AFX_ERR_UNKNOWN"
+
+
+def test_workspace_bytes_rejects_bad_sizes():
+    assert afx.afx_workspace_bytes(4096, 1) > 0
+    assert afx.afx_workspace_bytes(0, 1) == 0
+    assert afx.afx_workspace_bytes(4096, 9) == 0
+
+
+FAKE = 0x7F0000000000  # never dereferenced: validation fails first
+
+
+def _status(fn, *args):
+    with pytest.raises(afx.AfxError) as e:
+        fn(*args, stream=0)
+    return e.value.status
+
+
+def test_select_rejects_bad_arguments_on_the_host():
+    ok = dict(x=FAKE, dtype=0, K=64, T=1, mode=0, k=8, tau=0.0, idx=FAKE, count=FAKE)
+
+    def call(**kw):
+        a = {**ok, **kw}
+        return _status(afx.afx_select_active, a["x"], a["dtype"], a["K"], a["T"], a["mode"], a["k"],
+                       a["tau"], a["idx"], a["count"], None)
+
+    assert call(x=None) == 1 and call(idx=None) == 1 and call(count=None) == 1
+    assert call(K=0) == 1 and call(T=0) == 1 and call(T=9) == 1
+    assert call(k=-1) == 1 and call(k=65) == 1
+    assert call(dtype=7) == 4 and call(mode=3) == 4
+    assert call(x=FAKE + 1) == 2 and call(idx=FAKE + 2) == 2
+    assert call(mode=1, tau=float("nan")) == 1
+
+
+def test_gemv_rejects_bad_arguments_on_the_host():
+    ok = dict(Wt=FAKE, dtype=1, K=64, N=32, ldw=32, x=FAKE, T=1, idx=FAKE, count=FAKE, slot=None,
+              y=FAKE, acc=0, ws=FAKE)
+
+    def call(**kw):
+        a = {**ok, **kw}
+        return _status(afx.afx_sparse_gemv, a["Wt"], a["dtype"], a["K"], a["N"], a["ldw"], a["x"],
+                       a["T"], a["idx"], a["count"], a["slot"], a["y"], a["acc"], a["ws"])
+
+    for name in ("Wt", "x", "idx", "count", "y", "ws"):
+        assert call(**{name: None}) == 1
+    assert call(K=0) == 1 and call(N=0) == 1 and call(T=0) == 1 and call(T=9) == 1
+    assert call(ldw=24) == 1                       # ldw < N
+    assert call(dtype=2) == 4
+    assert call(N=36, ldw=40) == 2                 # N not a multiple of 8
+    assert call(ldw=36) == 2                       # ldw not a multiple of 8
+    assert call(Wt=FAKE + 8) == 2 and call(y=FAKE + 4) == 2 and call(ws=FAKE + 16) == 2
+    assert call(N=8 * 40000, ldw=8 * 40000) == 3   # more column tiles than the workspace counts
+
+
+def test_diff_rejects_bad_arguments_on_the_host():
+    assert _status(afx.afx_diff_active, None, FAKE, FAKE, 8, FAKE, FAKE, FAKE) == 1
+    assert _status(afx.afx_diff_active, FAKE, FAKE, FAKE, 0, FAKE, FAKE, FAKE) == 1

@@ -1,0 +1,141 @@
+"""GPU parity: afx_sparse_gemv against the fp64 oracle (max relative error 2e-3)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2504_08378_b200 import afx, synth
+from gpu_util import dev_bits, dev_i32, rel_err
+
+pytestmark = pytest.mark.gpu
+
+TOL = 2e-3  # max_i |y_i - ref_i| / max(|ref_i|, rms(ref)), fp32 sums vs fp64
+
+
+def run_gemv(Wt_bits, dt, N, x_bits, idx, slot=None, y0=None, ws=None):
+    x_bits = np.atleast_2d(x_bits)
+    T, K = x_bits.shape
+    ldw = Wt_bits.shape[1]
+    W, x = dev_bits(Wt_bits), dev_bits(x_bits)
+    cap = max(K, 1)
+    idx_d = torch.zeros((cap,), dtype=torch.int32, device="cuda")
+    idx_d[: len(idx)] = dev_i32(idx)
+    cnt = dev_i32([len(idx)])
+    slot_d = None
+    if slot is not None:
+        slot_d = torch.zeros((cap,), dtype=torch.int32, device="cuda")
+        slot_d[: len(slot)] = dev_i32(slot)
+    ws = afx.new_workspace(N, T) if ws is None else ws
+    if y0 is None:
+        y = torch.full((T, N), float("nan"), dtype=torch.float32, device="cuda")
+        acc = 0
+    else:
+        y = torch.from_numpy(np.ascontiguousarray(y0, np.float32)).cuda()
+        acc = 1
+    afx.afx_sparse_gemv(W, dt, K, N, ldw, x, T, idx_d, cnt, slot_d, y, acc, ws)
+    torch.cuda.synchronize()
+    return y.cpu().numpy()
+
+
+SHAPES = [  # K, N, ldw
+    (8, 8, 8), (31, 24, 24), (64, 264, 272), (512, 1376, 1376), (1000, 4096, 4096),
+    (4096, 2048 + 40, 2048 + 40), (2048, 11008, 11008),
+]
+
+
+@pytest.mark.parametrize("dt", ["f16", "bf16"])
+@pytest.mark.parametrize("K,N,ldw", SHAPES)
+def test_gemv_matches_oracle_at_several_sparsities(dt, K, N, ldw):
+    Wt = synth.weight(201, K * 7 + N, K, N, dt, ldw=ldw)
+    x = synth.laplace_bits(202, K, (K,), dt)
+    for k in sorted({0, 1, synth.keep_count(K, 50), synth.keep_count(K, 90), K}):
+        idx = oracle.select_active(x, dt, oracle.TOPK, k=k)
+        y = run_gemv(Wt, dt, N, x, idx)
+        ref = oracle.sparse_gemv(Wt, dt, N, x, idx)
+        assert y.shape == ref.shape and np.isfinite(y).all()
+        assert rel_err(y, ref) <= TOL, (K, N, k, rel_err(y, ref))
+        if k == 0:
+            assert (y == 0).all()
+
+
+def test_config1_single_projection():
+    """W fp16 512x1376, x Laplace(0,1), keep the top 50% of channels."""
+    dt, K, N = "f16", 512, 1376
+    Wt = synth.weight(1, 1, K, N, dt)
+    x = synth.laplace_bits(1, 2, (K,), dt)
+    x_d = dev_bits(x)
+    idx_d = torch.zeros(K, dtype=torch.int32, device="cuda")
+    cnt_d = torch.zeros(1, dtype=torch.int32, device="cuda")
+    afx.afx_select_active(x_d, dt, K, 1, afx.MODE_TOPK, 256, 0.0, idx_d, cnt_d)
+    idx = oracle.select_active(x, dt, oracle.TOPK, k=256)
+    assert int(cnt_d.item()) == 256 and np.array_equal(idx_d.cpu().numpy()[:256], idx)
+    y = torch.empty((1, N), dtype=torch.float32, device="cuda")
+    ws = afx.new_workspace(N, 1)
+    afx.afx_sparse_gemv(dev_bits(Wt), dt, K, N, N, x_d, 1, idx_d, cnt_d, None, y, 0, ws)
+    torch.cuda.synchronize()
+    assert rel_err(y.cpu().numpy(), oracle.sparse_gemv(Wt, dt, N, x, idx)) <= TOL
+
+
+@pytest.mark.parametrize("dt", ["f16", "bf16"])
+@pytest.mark.parametrize("T", [2, 3, 4, 8])
+def test_multi_token_union(dt, T):
+    K, N = 1536, 2304 + 8
+    Wt = synth.weight(203, T, K, N, dt)
+    x = synth.laplace_bits(204, T, (T, K), dt)
+    idx = oracle.select_active(x, dt, oracle.TOPK, k=synth.keep_count(K, 60))
+    y = run_gemv(Wt, dt, N, x, idx)
+    ref = oracle.sparse_gemv(Wt, dt, N, x, idx)
+    assert rel_err(y, ref) <= TOL
+
+
+def test_accumulate_adds_to_y_and_workspace_is_reusable():
+    dt, K, N = "bf16", 2048, 4096
+    Wt = synth.weight(205, 1, K, N, dt)
+    x = synth.laplace_bits(205, 2, (K,), dt)
+    idx = oracle.select_active(x, dt, oracle.THRESHOLD, tau=synth.laplace_tau(0.5))
+    ref = oracle.sparse_gemv(Wt, dt, N, x, idx)
+    y0 = synth.laplace(205, 3, (1, N)).astype(np.float32)
+    ws = afx.new_workspace(N, 1)
+    for _ in range(3):  # the same workspace, call after call
+        y = run_gemv(Wt, dt, N, x, idx, y0=y0, ws=ws)
+        assert rel_err(y, ref + y0) <= TOL
+    y_a = run_gemv(Wt, dt, N, x, idx, ws=ws)
+    y_b = run_gemv(Wt, dt, N, x, idx, ws=ws)
+    assert np.array_equal(y_a, y_b), "sums must not depend on block timing"
+
+
+def test_slot_list_reads_columns_from_a_cache():
+    dt, K, N = "f16", 600, 520
+    Wt = synth.weight(206, 1, K, N, dt)
+    x = synth.laplace_bits(206, 2, (K,), dt)
+    idx = oracle.select_active(x, dt, oracle.TOPK, k=200)
+    perm = np.random.default_rng(1).permutation(idx.size).astype(np.int32)
+    cache = np.zeros((idx.size, N), np.uint16)
+    cache[perm] = Wt[idx]                              # column idx[c] lives in slot perm[c]
+    y = run_gemv(cache, dt, N, x, idx, slot=perm)
+    assert rel_err(y, oracle.sparse_gemv(Wt, dt, N, x, idx)) <= TOL
+
+
+def test_dense_equals_sparse_when_dropped_channels_are_zero():
+    dt, K, N = "bf16", 1024, 1024
+    Wt = synth.weight(207, 1, K, N, dt)
+    x = synth.laplace_bits(207, 2, (K,), dt)
+    idx = oracle.select_active(x, dt, oracle.TOPK, k=300)
+    xz = np.zeros_like(x)
+    xz[idx] = x[idx]
+    dense = run_gemv(Wt, dt, N, xz, np.arange(K))
+    sparse = run_gemv(Wt, dt, N, x, idx)
+    assert rel_err(dense, sparse.astype(np.float64)) <= 1e-5
+
+
+def test_integer_weights_give_exact_results():
+    g = np.random.default_rng(6)
+    K, N = 300, 264
+    W = g.integers(-8, 9, (K, N)).astype(np.float32)
+    xv = g.integers(-8, 9, K).astype(np.float32)
+    for dt in ("f16", "bf16"):
+        idx = np.sort(g.choice(K, 120, replace=False)).astype(np.int32)
+        y = run_gemv(synth.f32_to_bits(W, dt), dt, N, synth.f32_to_bits(xv, dt), idx)
+        assert np.array_equal(y[0].astype(np.float64),
+                              oracle.sparse_gemv(synth.f32_to_bits(W, dt), dt, N,
+                                                 synth.f32_to_bits(xv, dt), idx)[0])
