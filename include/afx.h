@@ -55,19 +55,6 @@ afx_status afx_version(int* major, int* minor);
 const char* afx_status_string(afx_status s);
 
 /*
- * Scratch memory needed by afx_sparse_gemv for operators of at most N_max outputs and T_max
- * tokens on the current device.  The caller allocates that many bytes of DEVICE memory
- * (256-byte aligned) once, clears it with afx_workspace_init before its first use, and may
- * reuse it for any number of calls that are ordered on one stream.  Two calls that may
- * overlap on the GPU need two workspaces.  Returns 0 on a bad argument.
- */
-size_t afx_workspace_bytes(int N_max, int T_max);
-
-/* Enqueue the clearing of a fresh workspace (its split counters must start at zero;
- * every call leaves them at zero again). */
-afx_status afx_workspace_init(void* workspace /*DEVICE*/, size_t bytes, void* stream);
-
-/*
  * Active-channel selection ("Top-K" operation T of the swapping pipeline, Sec. 4; the
  * magnitude rule of Sec. 2.1; the index-generating kernel of Sec. 6 "Caching").
  *
@@ -105,18 +92,121 @@ afx_status afx_diff_active(const int32_t* idxA, const int32_t* cntA, const uint3
  *
  * with col(c) = idx[c], or slot[c] when `slot` is given (the columns then live in a cache
  * whose slot list afx_cache_fetch produced).  Products are exact in fp32; sums are fp32 in
- * a fixed order (same inputs give the same bits).
+ * a fixed order (same inputs on the same device give the same bits).
  *
  *   Wt        DEVICE, channel-contiguous weights (see the conventions above).
  *   x         DEVICE, [T][K] 16-bit floats; every token uses the whole list.
  *   idx,count DEVICE; entries must lie in [0,K) (not checked on the device).
  *   slot      DEVICE int32[*count] or NULL.
  *   y         DEVICE, [T][N] fp32, 16-byte aligned.  accumulate = 0 overwrites, 1 adds.
- *   workspace DEVICE scratch from afx_workspace_bytes(N, T), initialised once.
+ * Needs no scratch memory.  N <= 4 194 240.
  */
 afx_status afx_sparse_gemv(const void* Wt, int dtype, int K, int N, int64_t ldw, const void* x,
                            int T, const int32_t* idx, const int32_t* count, const int32_t* slot,
-                           float* y, int accumulate, void* workspace, void* stream);
+                           float* y, int accumulate, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Decoder layers: every linear operator of a Llama-shaped layer run as ONE kernel that
+ * normalises (where the layer does), selects the active channels of its own input and
+ * evaluates the operator on them -- the paper's per-operator T (Top-K) + C (compute) pair of
+ * Sec. 4 applied "to all linear transformation operators" (Sec. 2.1), with the cross-layer
+ * prediction and miss bookkeeping of Sec. 3.  Attention itself stays dense.
+ * ------------------------------------------------------------------------------------------ */
+
+typedef struct afx_model afx_model; /* opaque, HOST object */
+typedef struct afx_state afx_state; /* opaque, HOST object describing a DEVICE blob */
+
+/* The four distinct operator inputs of a layer (q, k and v share one; gate and up share one). */
+#define AFX_OP_QKV 0  /* input: RMSNorm(h) * g_attn        -> q | k | v          */
+#define AFX_OP_O 1    /* input: attention output           -> h += W_o a         */
+#define AFX_OP_GU 2   /* input: RMSNorm(h) * g_mlp         -> silu(gate) * up    */
+#define AFX_OP_DOWN 3 /* input: silu(gate) * up            -> h += W_down hm     */
+
+#define AFX_XL_OFF 0      /* no cross-layer prediction                                         */
+#define AFX_XL_BOOKKEEP 1 /* paper: compute on the actual set A; the set P predicted by an    */
+                          /* earlier layer only decides what was preloaded; A \ P is listed    */
+#define AFX_XL_REUSE 2    /* compute on the predicted set P, no selection in predicted layers  */
+
+typedef struct {
+    int32_t dtype;       /* AFX_F16 / AFX_BF16: weights and rounded activations               */
+    int32_t n_layers;
+    int32_t hidden;      /* model width; multiple of 8                                         */
+    int32_t n_heads;     /* query heads                                                        */
+    int32_t n_kv_heads;  /* divides n_heads, n_heads / n_kv_heads <= 8                         */
+    int32_t head_dim;    /* must be 128                                                        */
+    int32_t mlp;         /* MLP width; multiple of 8                                           */
+    int32_t max_seq;     /* rows of each KV cache; positions 0 .. max_seq-1                    */
+    float rms_eps;
+    float rope_theta;
+    int32_t select_mode; /* AFX_MODE_TOPK / AFX_MODE_THRESHOLD                                 */
+    int32_t xl_depth;    /* d: layers p = 0, d, 2d, .. predict layers p+1 .. p+d; 0 = off      */
+    int32_t xl_mode;     /* AFX_XL_*                                                           */
+} afx_model_desc;
+
+typedef struct {
+    /* DEVICE pointers, channel-contiguous (see the conventions at the top), 16-byte aligned:  */
+    const void* w_qkv;  /* [hidden][(n_heads + 2 n_kv_heads) * 128]  columns: q | k | v        */
+    const void* w_o;    /* [n_heads * 128][hidden]                                             */
+    const void* w_gu;   /* [hidden][2 * mlp]: columns in groups of 16 = gate[8m..8m+8) then    */
+                        /* up[8m..8m+8), so that one pass yields silu(gate) * up               */
+    const void* w_down; /* [mlp][hidden]                                                       */
+    const float* g_attn; /* [hidden] fp32 RMSNorm gains                                        */
+    const float* g_mlp;
+    void* k_cache;      /* [T][max_seq][n_kv_heads][128] fp16, one cache per token stream      */
+    void* v_cache;
+    int32_t k[4];       /* per AFX_OP_*: channels kept in top-k mode                           */
+    float tau[4];       /* per AFX_OP_*: threshold in threshold mode                           */
+} afx_layer_desc;
+
+/*
+ * Creates the HOST-side model object: copies both descriptor arrays (layers[n_layers]) and
+ * allocates one small DEVICE table (rotary cos/sin, 512 * max_seq bytes) with cudaMalloc.
+ * Weights and caches stay the caller's.  afx_model_destroy frees the table and the object.
+ */
+afx_status afx_model_create(const afx_model_desc* desc, const afx_layer_desc* layers, afx_model** out);
+afx_status afx_model_destroy(afx_model* model);
+
+/*
+ * Per-sequence working set for T token streams decoded together (1 <= T <= AFX_MAX_T): the
+ * fp32 residual h[T][hidden], the operators' intermediate vectors, the current and predicted
+ * active sets of the four operator inputs, and per-layer counters.  The caller allocates
+ * afx_state_bytes() of DEVICE memory (256-byte aligned); afx_state_create clears it on
+ * `stream` and returns a HOST handle that only records where things live in the blob.
+ */
+size_t afx_state_bytes(const afx_model* model, int T);
+afx_status afx_state_create(const afx_model* model, int T, void* blob, size_t bytes, void* stream,
+                            afx_state** out);
+afx_status afx_state_destroy(afx_state* state);
+
+/* Buffers inside the state blob (DEVICE addresses), for loading h and reading results back. */
+#define AFX_BUF_H 0          /* fp32 [T][hidden]      residual stream, input and output       */
+#define AFX_BUF_QKV 1        /* fp32 [T][n_qkv]       q | k | v before rotation               */
+#define AFX_BUF_ATTN 2       /* dtype [T][n_heads*128] attention output (input of W_o)         */
+#define AFX_BUF_HM 3         /* dtype [T][mlp]        silu(gate)*up (input of W_down)          */
+#define AFX_BUF_XNORM 4      /* dtype [T][hidden]     op = AFX_OP_QKV or AFX_OP_GU: normed input */
+#define AFX_BUF_IDX 5        /* int32 [K_op]          active list last used by operator input `op` */
+#define AFX_BUF_MISS 6       /* int32 [K_op]          A \ P of the last bookkeeping            */
+#define AFX_BUF_STATS 7      /* int32 [n_layers][4][4] per layer and op: list length, |A & P|,  */
+                             /*                       |A \ P|, 0 (written by each layer step)  */
+afx_status afx_state_buffer(const afx_state* state, int which, int op, void** ptr, size_t* bytes);
+
+/*
+ * One decoder layer for the T token streams at position `pos` (0 <= pos < max_seq; the
+ * cache rows 0..pos-1 hold the past, row pos is written): five kernels on `stream`,
+ *   qkv (RMSNorm + select + GEMV) -> rotary, cache append, dense attention ->
+ *   o (select + GEMV, h +=) -> gate/up (RMSNorm + select + GEMV + silu*up) ->
+ *   down (select + GEMV, h +=).
+ * Layers must be stepped in order 0 .. n_layers-1 when cross-layer prediction is on.
+ */
+afx_status afx_layer_step(afx_model* model, int layer, afx_state* state, int pos, void* stream);
+
+/*
+ * The MLP block alone on a given (already normalised) input: y = W_down(silu(W_gate x) * W_up x)
+ * with both selections; x DEVICE [T][hidden] dtype, y DEVICE [T][hidden] fp32 (overwritten).
+ * Uses the state's HM buffer and active-set buffers; no cross-layer prediction.
+ */
+afx_status afx_mlp_block(afx_model* model, int layer, afx_state* state, const void* x, float* y,
+                         void* stream);
 
 #ifdef __cplusplus
 }

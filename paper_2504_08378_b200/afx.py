@@ -13,6 +13,9 @@ from ctypes import c_float, c_int, c_int32, c_int64, c_size_t, c_void_p
 from . import build as _build
 
 F16, BF16 = 0, 1
+OP_QKV, OP_O, OP_GU, OP_DOWN = 0, 1, 2, 3
+XL_OFF, XL_BOOKKEEP, XL_REUSE = 0, 1, 2
+BUF_H, BUF_QKV, BUF_ATTN, BUF_HM, BUF_XNORM, BUF_IDX, BUF_MISS, BUF_STATS = range(8)
 MODE_TOPK, MODE_THRESHOLD = 0, 1
 MAX_T = 8
 DTYPES = {"f16": F16, "bf16": BF16}
@@ -21,6 +24,21 @@ STATUS_NAMES = {
     0: "AFX_OK", 1: "AFX_ERR_INVALID_ARG", 2: "AFX_ERR_ALIGNMENT", 3: "AFX_ERR_CAPACITY",
     4: "AFX_ERR_UNSUPPORTED", 5: "AFX_ERR_CUDA", 6: "AFX_ERR_TIMEOUT",
 }
+
+
+class ModelDesc(ctypes.Structure):
+    """afx_model_desc"""
+    _fields_ = [("dtype", c_int32), ("n_layers", c_int32), ("hidden", c_int32), ("n_heads", c_int32),
+                ("n_kv_heads", c_int32), ("head_dim", c_int32), ("mlp", c_int32), ("max_seq", c_int32),
+                ("rms_eps", c_float), ("rope_theta", c_float), ("select_mode", c_int32),
+                ("xl_depth", c_int32), ("xl_mode", c_int32)]
+
+
+class LayerDesc(ctypes.Structure):
+    """afx_layer_desc"""
+    _fields_ = [("w_qkv", c_void_p), ("w_o", c_void_p), ("w_gu", c_void_p), ("w_down", c_void_p),
+                ("g_attn", c_void_p), ("g_mlp", c_void_p), ("k_cache", c_void_p), ("v_cache", c_void_p),
+                ("k", c_int32 * 4), ("tau", c_float * 4)]
 
 
 class AfxError(RuntimeError):
@@ -41,16 +59,24 @@ def lib() -> ctypes.CDLL:
         L.afx_version.argtypes = [ctypes.POINTER(c_int), ctypes.POINTER(c_int)]
         L.afx_status_string.restype = ctypes.c_char_p
         L.afx_status_string.argtypes = [c_int32]
-        L.afx_workspace_bytes.restype = c_size_t
-        L.afx_workspace_bytes.argtypes = [c_int, c_int]
-        L.afx_workspace_init.argtypes = [c_void_p, c_size_t, c_void_p]
         L.afx_select_active.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_int, c_float,
                                         c_void_p, c_void_p, c_void_p, c_void_p]
         L.afx_diff_active.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p,
                                       c_void_p, c_void_p]
         L.afx_sparse_gemv.argtypes = [c_void_p, c_int, c_int, c_int, c_int64, c_void_p, c_int,
-                                      c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p,
-                                      c_void_p]
+                                      c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p]
+        L.afx_model_create.argtypes = [ctypes.POINTER(ModelDesc), ctypes.POINTER(LayerDesc),
+                                       ctypes.POINTER(c_void_p)]
+        L.afx_model_destroy.argtypes = [c_void_p]
+        L.afx_state_bytes.restype = c_size_t
+        L.afx_state_bytes.argtypes = [c_void_p, c_int]
+        L.afx_state_create.argtypes = [c_void_p, c_int, c_void_p, c_size_t, c_void_p,
+                                       ctypes.POINTER(c_void_p)]
+        L.afx_state_destroy.argtypes = [c_void_p]
+        L.afx_state_buffer.argtypes = [c_void_p, c_int, c_int, ctypes.POINTER(c_void_p),
+                                       ctypes.POINTER(c_size_t)]
+        L.afx_layer_step.argtypes = [c_void_p, c_int, c_void_p, c_int, c_void_p]
+        L.afx_mlp_block.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p]
         _lib = L
     return _lib
 
@@ -91,14 +117,6 @@ def afx_status_string(status: int) -> str:
     return lib().afx_status_string(int(status)).decode()
 
 
-def afx_workspace_bytes(N_max: int, T_max: int = 1) -> int:
-    return int(lib().afx_workspace_bytes(int(N_max), int(T_max)))
-
-
-def afx_workspace_init(workspace, nbytes: int, stream=None):
-    _check("afx_workspace_init", lib().afx_workspace_init(_ptr(workspace), int(nbytes), _stream(stream)))
-
-
 def afx_select_active(x, dtype, K: int, T: int, mode: int, k: int, tau: float, idx, count,
                       bitmap=None, stream=None):
     _check("afx_select_active",
@@ -113,21 +131,50 @@ def afx_diff_active(idxA, cntA, bitmapP, K: int, miss, miss_count, hit_count, st
 
 
 def afx_sparse_gemv(Wt, dtype, K: int, N: int, ldw: int, x, T: int, idx, count, slot, y,
-                    accumulate: int, workspace, stream=None):
+                    accumulate: int, stream=None):
     _check("afx_sparse_gemv",
            lib().afx_sparse_gemv(_ptr(Wt), _dt(dtype), int(K), int(N), int(ldw), _ptr(x), int(T),
                                  _ptr(idx), _ptr(count), _ptr(slot), _ptr(y), int(accumulate),
-                                 _ptr(workspace), _stream(stream)))
+                                 _stream(stream)))
 
 
-def new_workspace(N_max: int, T_max: int = 1, device="cuda", stream=None):
-    """Allocates (torch) and clears a GEMV workspace; returns the uint8 tensor."""
-    import torch
-    n = afx_workspace_bytes(N_max, T_max)
-    if n == 0:
-        raise AfxError("afx_workspace_bytes", 1)
-    ws = torch.empty(n + 256, dtype=torch.uint8, device=device)
-    off = (-ws.data_ptr()) % 256
-    ws = ws[off:off + n]
-    afx_workspace_init(ws, n, stream)
-    return ws
+def afx_model_create(desc: ModelDesc, layers) -> int:
+    """layers: sequence of LayerDesc (len == desc.n_layers).  Returns the model handle."""
+    arr = (LayerDesc * len(layers))(*layers)
+    out = c_void_p(0)
+    _check("afx_model_create", lib().afx_model_create(ctypes.byref(desc), arr, ctypes.byref(out)))
+    return out.value
+
+
+def afx_model_destroy(model: int):
+    _check("afx_model_destroy", lib().afx_model_destroy(model))
+
+
+def afx_state_bytes(model: int, T: int) -> int:
+    return int(lib().afx_state_bytes(model, int(T)))
+
+
+def afx_state_create(model: int, T: int, blob, nbytes: int, stream=None) -> int:
+    out = c_void_p(0)
+    _check("afx_state_create",
+           lib().afx_state_create(model, int(T), _ptr(blob), int(nbytes), _stream(stream), ctypes.byref(out)))
+    return out.value
+
+
+def afx_state_destroy(state: int):
+    _check("afx_state_destroy", lib().afx_state_destroy(state))
+
+
+def afx_state_buffer(state: int, which: int, op: int = 0):
+    """Returns (device address, bytes) of a buffer inside the state blob."""
+    ptr, n = c_void_p(0), c_size_t(0)
+    _check("afx_state_buffer", lib().afx_state_buffer(state, int(which), int(op), ctypes.byref(ptr), ctypes.byref(n)))
+    return ptr.value, n.value
+
+
+def afx_layer_step(model: int, layer: int, state: int, pos: int, stream=None):
+    _check("afx_layer_step", lib().afx_layer_step(model, int(layer), state, int(pos), _stream(stream)))
+
+
+def afx_mlp_block(model: int, layer: int, state: int, x, y, stream=None):
+    _check("afx_mlp_block", lib().afx_mlp_block(model, int(layer), state, _ptr(x), _ptr(y), _stream(stream)))

@@ -1,30 +1,20 @@
-// afx_sparse_gemv and its workspace.
-#include "afx_gemv.cuh"
+// afx_sparse_gemv: host-side shape selection and launch.
+#include "afx_launch.cuh"
 
 namespace afx {
 
-// Launch shapes.  512 threads per block; tokens decide the register budget and with it how
-// many blocks stay resident per SM.
-constexpr int kGemvWN = 1;
-constexpr int kGemvWC = 16;
-constexpr int kGemvThreads = 32 * kGemvWN * kGemvWC;
-constexpr int kGemvUnroll = 8;
-constexpr int kCountersBytes = 4096;  // room for 1024 tile counters
-
 template <int TMAX>
 struct GemvShape {
-    static constexpr int kBlocksPerSM = TMAX <= 2 ? 2 : 1;
+    static constexpr int kBlocksPerSM = TMAX <= 1 ? 2 : 1;
     static constexpr int kStageCap = TMAX <= 4 ? 1024 : 512;
 };
 
-template <int DT, int TMAX>
+template <int DT, int TMAX, int PW>
 __global__ void __launch_bounds__(kGemvThreads, GemvShape<TMAX>::kBlocksPerSM)
-sparse_gemv_kernel(GemvArgs a) {
+sparse_gemv_kernel(GemvListArgs a) {
     constexpr int CAP = GemvShape<TMAX>::kStageCap;
-    __shared__ GemvShared<CAP> sh;
-    __shared__ float s_x[TMAX * CAP];
-    __shared__ __align__(16) float s_red[kGemvWC * kGemvWN * kPieceW];
-    gemv_block<DT, TMAX, kGemvWN, kGemvWC, kGemvUnroll, CAP>(a, &sh, s_x, s_red);
+    __shared__ GemvSmem<TMAX, CAP> sm;
+    gemv_list_block<DT, TMAX, PW, CAP>(a, &sm);
 }
 
 int sm_count() {
@@ -39,61 +29,50 @@ int sm_count() {
     return cached[dev];
 }
 
-static int gemv_grid(int tmax) {
-    const int per_sm = tmax <= 2 ? 2 : 1;
-    return sm_count() * per_sm;
+int g_force_pw = 0, g_force_s = 0;  // experiment knobs, 0 = automatic
+
+template <int DT, int TMAX>
+static afx_status launch_gemv_t(const GemvListArgs& a, cudaStream_t st) {
+    const void* kerns[3] = {reinterpret_cast<const void*>(sparse_gemv_kernel<DT, TMAX, 256>),
+                            reinterpret_cast<const void*>(sparse_gemv_kernel<DT, TMAX, 128>),
+                            reinterpret_cast<const void*>(sparse_gemv_kernel<DT, TMAX, 64>)};
+    const GemvShapeChoice c = choose_gemv_shape(a.N, kerns, 0, g_force_pw, g_force_s);
+    switch (c.pw) {
+        case 256: return launch_clustered(sparse_gemv_kernel<DT, TMAX, 256>, c.S, c.tiles, 0, a, st);
+        case 128: return launch_clustered(sparse_gemv_kernel<DT, TMAX, 128>, c.S, c.tiles, 0, a, st);
+        default: return launch_clustered(sparse_gemv_kernel<DT, TMAX, 64>, c.S, c.tiles, 0, a, st);
+    }
 }
 
-static int tmax_for(int T) { return T <= 1 ? 1 : (T <= 2 ? 2 : (T <= 4 ? 4 : 8)); }
-
 template <int DT>
-static afx_status launch_gemv(const GemvArgs& a, cudaStream_t st) {
-    const int tmax = tmax_for(a.T);
-    const int grid = gemv_grid(tmax);
-    if (grid <= 0) return AFX_ERR_CUDA;
-    switch (tmax) {
-        case 1: sparse_gemv_kernel<DT, 1><<<grid, kGemvThreads, 0, st>>>(a); break;
-        case 2: sparse_gemv_kernel<DT, 2><<<grid, kGemvThreads, 0, st>>>(a); break;
-        case 4: sparse_gemv_kernel<DT, 4><<<grid, kGemvThreads, 0, st>>>(a); break;
-        default: sparse_gemv_kernel<DT, 8><<<grid, kGemvThreads, 0, st>>>(a); break;
-    }
-    return launch_status();
+static afx_status launch_gemv(const GemvListArgs& a, cudaStream_t st) {
+    if (a.T <= 1) return launch_gemv_t<DT, 1>(a, st);
+    if (a.T <= 2) return launch_gemv_t<DT, 2>(a, st);
+    if (a.T <= 4) return launch_gemv_t<DT, 4>(a, st);
+    return launch_gemv_t<DT, 8>(a, st);
 }
 
 }  // namespace afx
 
-extern "C" size_t afx_workspace_bytes(int N_max, int T_max) {
-    using namespace afx;
-    if (N_max <= 0 || T_max < 1 || T_max > AFX_MAX_T) return 0;
-    const int sms = sm_count();
-    const size_t blocks = static_cast<size_t>(sms > 0 ? sms : 256) * 2;
-    const size_t tiles = static_cast<size_t>(N_max + kPieceW - 1) / kPieceW;
-    if (tiles * sizeof(int) > kCountersBytes) return 0;
-    return kCountersBytes + (blocks + tiles) * static_cast<size_t>(T_max) * kGemvWN * kPieceW * sizeof(float);
-}
-
-extern "C" afx_status afx_workspace_init(void* workspace, size_t bytes, void* stream) {
-    if (workspace == nullptr || bytes < afx::kCountersBytes) return AFX_ERR_INVALID_ARG;
-    if (cudaMemsetAsync(workspace, 0, afx::kCountersBytes, static_cast<cudaStream_t>(stream)) != cudaSuccess)
-        return AFX_ERR_CUDA;
-    return AFX_OK;
+// Not part of the ABI: forces tile width / cluster size for kernel experiments (0 = automatic).
+extern "C" void afx_internal_tune_gemv(int pw, int s) {
+    afx::g_force_pw = pw;
+    afx::g_force_s = s;
 }
 
 extern "C" afx_status afx_sparse_gemv(const void* Wt, int dtype, int K, int N, int64_t ldw,
                                       const void* x, int T, const int32_t* idx, const int32_t* count,
-                                      const int32_t* slot, float* y, int accumulate, void* workspace,
-                                      void* stream) {
+                                      const int32_t* slot, float* y, int accumulate, void* stream) {
     using namespace afx;
-    if (Wt == nullptr || x == nullptr || idx == nullptr || count == nullptr || y == nullptr ||
-        workspace == nullptr)
+    if (Wt == nullptr || x == nullptr || idx == nullptr || count == nullptr || y == nullptr)
         return AFX_ERR_INVALID_ARG;
     if (K <= 0 || N <= 0 || T < 1 || T > AFX_MAX_T || ldw < N) return AFX_ERR_INVALID_ARG;
     if (dtype != AFX_F16 && dtype != AFX_BF16) return AFX_ERR_UNSUPPORTED;
     if ((N & 7) != 0 || (ldw & 7) != 0 || !aligned16(Wt) || !aligned16(y) ||
-        (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0 || (reinterpret_cast<uintptr_t>(x) & 1u) != 0)
+        (reinterpret_cast<uintptr_t>(x) & 1u) != 0)
         return AFX_ERR_ALIGNMENT;
-    if (static_cast<size_t>(N + kPieceW - 1) / kPieceW * sizeof(int) > kCountersBytes) return AFX_ERR_CAPACITY;
-    GemvArgs a;
+    if ((N + 63) / 64 > 65535) return AFX_ERR_CAPACITY;
+    GemvListArgs a;
     a.Wt = static_cast<const uint16_t*>(Wt);
     a.ldw = ldw;
     a.K = K;
@@ -103,10 +82,10 @@ extern "C" afx_status afx_sparse_gemv(const void* Wt, int dtype, int K, int N, i
     a.idx = idx;
     a.count = count;
     a.slot = slot;
-    a.y = y;
     a.accumulate = accumulate ? 1 : 0;
-    a.counters = static_cast<int*>(workspace);
-    a.partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + kCountersBytes);
+    a.ep.y = y;
+    a.ep.out_bits = nullptr;
+    a.ep.N = N;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     return dtype == AFX_F16 ? launch_gemv<AFX_F16>(a, st) : launch_gemv<AFX_BF16>(a, st);
 }

@@ -1,0 +1,427 @@
+// afx_model_* / afx_state_* / afx_layer_step / afx_mlp_block: a decoder layer as five kernels.
+#include <math.h>
+#include <new>
+#include <vector>
+
+#include "afx_attn.cuh"
+#include "afx_fused.cuh"
+#include "afx_launch.cuh"
+
+namespace afx {
+
+template <int TMAX>
+struct FusedShape {
+    static constexpr int kBlocksPerSM = TMAX <= 1 ? 2 : 1;
+    static constexpr int kStageCap = TMAX <= 4 ? 1024 : 512;
+};
+
+template <int DT, int TMAX, int PW, int IN, int EP>
+__global__ void __launch_bounds__(kGemvThreads, FusedShape<TMAX>::kBlocksPerSM)
+fused_op_kernel(FusedArgs a) {
+    constexpr int CAP = FusedShape<TMAX>::kStageCap;
+    extern __shared__ __align__(16) unsigned char dyn[];
+    __shared__ GemvSmem<TMAX, CAP> sm;
+    __shared__ SelectScratch sel;
+    fused_op_block<DT, TMAX, PW, CAP, IN, EP>(a, dyn, &sm, &sel);
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(AttnArgs a) {
+    __shared__ AttnSmem sm;
+    attention_block<DT>(a, &sm);
+}
+
+template <int DT, int TMAX, int IN, int EP>
+static afx_status launch_fused_t(const FusedArgs& a, cudaStream_t st) {
+    const size_t dyn = fused_dyn_smem(IN, a.K, a.T);
+    const void* kerns[3] = {reinterpret_cast<const void*>(fused_op_kernel<DT, TMAX, 256, IN, EP>),
+                            reinterpret_cast<const void*>(fused_op_kernel<DT, TMAX, 128, IN, EP>),
+                            reinterpret_cast<const void*>(fused_op_kernel<DT, TMAX, 64, IN, EP>)};
+    const GemvShapeChoice c = choose_gemv_shape(a.N, kerns, dyn, g_force_pw, g_force_s);
+    switch (c.pw) {
+        case 256: return launch_clustered(fused_op_kernel<DT, TMAX, 256, IN, EP>, c.S, c.tiles, dyn, a, st);
+        case 128: return launch_clustered(fused_op_kernel<DT, TMAX, 128, IN, EP>, c.S, c.tiles, dyn, a, st);
+        default: return launch_clustered(fused_op_kernel<DT, TMAX, 64, IN, EP>, c.S, c.tiles, dyn, a, st);
+    }
+}
+
+template <int DT, int IN, int EP>
+static afx_status launch_fused_dt(const FusedArgs& a, cudaStream_t st) {
+    if (a.T <= 1) return launch_fused_t<DT, 1, IN, EP>(a, st);
+    if (a.T <= 4) return launch_fused_t<DT, 4, IN, EP>(a, st);
+    return launch_fused_t<DT, 8, IN, EP>(a, st);
+}
+
+template <int IN, int EP>
+static afx_status launch_fused(int dtype, const FusedArgs& a, cudaStream_t st) {
+    return dtype == AFX_F16 ? launch_fused_dt<AFX_F16, IN, EP>(a, st) : launch_fused_dt<AFX_BF16, IN, EP>(a, st);
+}
+
+static afx_status launch_attention(int dtype, const AttnArgs& a, cudaStream_t st) {
+    // split the cached positions so that kv_heads * T * S blocks fill the machine, S <= 8
+    const int groups = a.kv_heads * a.T;
+    int S = (2 * sm_count() + groups - 1) / groups;
+    S = S < 1 ? 1 : (S > 8 ? 8 : S);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(S, a.kv_heads, a.T);
+    cfg.blockDim = dim3(kAttnThreads, 1, 1);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = S;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    const cudaError_t e = dtype == AFX_F16 ? cudaLaunchKernelEx(&cfg, attention_kernel<AFX_F16>, a)
+                                           : cudaLaunchKernelEx(&cfg, attention_kernel<AFX_BF16>, a);
+    return e == cudaSuccess ? AFX_OK : AFX_ERR_CUDA;
+}
+
+static size_t align256(size_t b) { return (b + 255) / 256 * 256; }
+
+}  // namespace afx
+
+struct afx_model {
+    afx_model_desc d;
+    std::vector<afx_layer_desc> layers;
+    float* rope = nullptr;  // DEVICE: cos[max_seq][64] then sin[max_seq][64]
+    int n_qkv = 0;
+    int K_op[4] = {0, 0, 0, 0};
+};
+
+struct afx_state {
+    const afx_model* model;
+    int T;
+    char* blob;
+    size_t bytes;
+    size_t off_h, off_qkv, off_attn, off_hm, off_xnorm[2], off_idx[4], off_miss[4], off_pred[4][2], off_stats;
+    size_t sz_h, sz_qkv, sz_attn, sz_hm, sz_xnorm, sz_idx[4], sz_pred[4], sz_stats;
+};
+
+static void state_layout(const afx_model* m, int T, afx_state* s) {
+    using afx::align256;
+    const afx_model_desc& d = m->d;
+    size_t o = 0;
+    auto take = [&](size_t bytes) {
+        const size_t at = o;
+        o += align256(bytes);
+        return at;
+    };
+    s->sz_h = static_cast<size_t>(T) * d.hidden * 4;
+    s->sz_qkv = static_cast<size_t>(T) * m->n_qkv * 4;
+    s->sz_attn = static_cast<size_t>(T) * d.n_heads * d.head_dim * 2;
+    s->sz_hm = static_cast<size_t>(T) * d.mlp * 2;
+    s->sz_xnorm = static_cast<size_t>(T) * d.hidden * 2;
+    s->off_h = take(s->sz_h);
+    s->off_qkv = take(s->sz_qkv);
+    s->off_attn = take(s->sz_attn);
+    s->off_hm = take(s->sz_hm);
+    s->off_xnorm[0] = take(s->sz_xnorm);
+    s->off_xnorm[1] = take(s->sz_xnorm);
+    for (int op = 0; op < 4; ++op) {
+        s->sz_idx[op] = static_cast<size_t>(m->K_op[op]) * 4;
+        s->sz_pred[op] = static_cast<size_t>((m->K_op[op] + 31) / 32) * 4;
+        s->off_idx[op] = take(s->sz_idx[op]);
+        s->off_miss[op] = take(s->sz_idx[op]);
+        s->off_pred[op][0] = take(s->sz_pred[op]);
+        s->off_pred[op][1] = take(s->sz_pred[op]);
+    }
+    s->sz_stats = static_cast<size_t>(d.n_layers) * 4 * 4 * 4;
+    s->off_stats = take(s->sz_stats);
+    s->bytes = o;
+}
+
+extern "C" afx_status afx_model_create(const afx_model_desc* desc, const afx_layer_desc* layers,
+                                       afx_model** out) {
+    using namespace afx;
+    if (desc == nullptr || layers == nullptr || out == nullptr) return AFX_ERR_INVALID_ARG;
+    const afx_model_desc& d = *desc;
+    if (d.dtype != AFX_F16 && d.dtype != AFX_BF16) return AFX_ERR_UNSUPPORTED;
+    if (d.select_mode != AFX_MODE_TOPK && d.select_mode != AFX_MODE_THRESHOLD) return AFX_ERR_UNSUPPORTED;
+    if (d.head_dim != kHeadDim) return AFX_ERR_UNSUPPORTED;
+    if (d.xl_mode < AFX_XL_OFF || d.xl_mode > AFX_XL_REUSE) return AFX_ERR_UNSUPPORTED;
+    if (d.n_layers < 1 || d.hidden < 8 || d.mlp < 8 || d.n_heads < 1 || d.n_kv_heads < 1 || d.max_seq < 1 ||
+        d.xl_depth < 0 || !(d.rms_eps >= 0.0f) || !(d.rope_theta > 0.0f))
+        return AFX_ERR_INVALID_ARG;
+    if (d.n_heads % d.n_kv_heads != 0 || d.n_heads / d.n_kv_heads > kAttnMaxRep) return AFX_ERR_UNSUPPORTED;
+    if ((d.hidden & 7) != 0 || (d.mlp & 7) != 0) return AFX_ERR_ALIGNMENT;
+    const int K_op[4] = {d.hidden, d.n_heads * d.head_dim, d.hidden, d.mlp};
+    for (int l = 0; l < d.n_layers; ++l) {
+        const afx_layer_desc& L = layers[l];
+        if (L.w_qkv == nullptr || L.w_o == nullptr || L.w_gu == nullptr || L.w_down == nullptr ||
+            L.g_attn == nullptr || L.g_mlp == nullptr || L.k_cache == nullptr || L.v_cache == nullptr)
+            return AFX_ERR_INVALID_ARG;
+        if (!aligned16(L.w_qkv) || !aligned16(L.w_o) || !aligned16(L.w_gu) || !aligned16(L.w_down) ||
+            !aligned16(L.k_cache) || !aligned16(L.v_cache))
+            return AFX_ERR_ALIGNMENT;
+        for (int op = 0; op < 4; ++op) {
+            if (d.select_mode == AFX_MODE_TOPK && (L.k[op] < 0 || L.k[op] > K_op[op])) return AFX_ERR_INVALID_ARG;
+            if (d.select_mode == AFX_MODE_THRESHOLD && L.tau[op] != L.tau[op]) return AFX_ERR_INVALID_ARG;
+        }
+    }
+    afx_model* m = new (std::nothrow) afx_model();
+    if (m == nullptr) return AFX_ERR_CAPACITY;
+    m->d = d;
+    m->layers.assign(layers, layers + d.n_layers);
+    m->n_qkv = (d.n_heads + 2 * d.n_kv_heads) * d.head_dim;
+    for (int op = 0; op < 4; ++op) m->K_op[op] = K_op[op];
+    // rotary table in fp64 on the host, stored as fp32
+    const int half = kHeadDim / 2;
+    std::vector<float> tab(static_cast<size_t>(2) * d.max_seq * half);
+    for (int p = 0; p < d.max_seq; ++p)
+        for (int i = 0; i < half; ++i) {
+            const double ang = static_cast<double>(p) * pow(static_cast<double>(d.rope_theta), -2.0 * i / kHeadDim);
+            tab[static_cast<size_t>(p) * half + i] = static_cast<float>(cos(ang));
+            tab[static_cast<size_t>(d.max_seq + p) * half + i] = static_cast<float>(sin(ang));
+        }
+    if (cudaMalloc(&m->rope, tab.size() * sizeof(float)) != cudaSuccess ||
+        cudaMemcpy(m->rope, tab.data(), tab.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) {
+        cudaGetLastError();
+        if (m->rope != nullptr) cudaFree(m->rope);
+        delete m;
+        return AFX_ERR_CUDA;
+    }
+    *out = m;
+    return AFX_OK;
+}
+
+extern "C" afx_status afx_model_destroy(afx_model* model) {
+    if (model == nullptr) return AFX_ERR_INVALID_ARG;
+    if (model->rope != nullptr) cudaFree(model->rope);
+    delete model;
+    return AFX_OK;
+}
+
+extern "C" size_t afx_state_bytes(const afx_model* model, int T) {
+    if (model == nullptr || T < 1 || T > AFX_MAX_T) return 0;
+    afx_state s;
+    state_layout(model, T, &s);
+    return s.bytes;
+}
+
+extern "C" afx_status afx_state_create(const afx_model* model, int T, void* blob, size_t bytes, void* stream,
+                                       afx_state** out) {
+    if (model == nullptr || blob == nullptr || out == nullptr || T < 1 || T > AFX_MAX_T) return AFX_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(blob) & 255u) != 0) return AFX_ERR_ALIGNMENT;
+    afx_state* s = new (std::nothrow) afx_state();
+    if (s == nullptr) return AFX_ERR_CAPACITY;
+    state_layout(model, T, s);
+    if (bytes < s->bytes) {
+        delete s;
+        return AFX_ERR_CAPACITY;
+    }
+    // the widest input stage must fit one block's shared memory
+    const size_t dyn_max = afx::fused_dyn_smem(afx::IN_NORM, model->d.hidden, T);
+    if (dyn_max > 160 * 1024) {
+        delete s;
+        return AFX_ERR_UNSUPPORTED;
+    }
+    s->model = model;
+    s->T = T;
+    s->blob = static_cast<char*>(blob);
+    if (cudaMemsetAsync(blob, 0, s->bytes, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        cudaGetLastError();
+        delete s;
+        return AFX_ERR_CUDA;
+    }
+    *out = s;
+    return AFX_OK;
+}
+
+extern "C" afx_status afx_state_destroy(afx_state* state) {
+    if (state == nullptr) return AFX_ERR_INVALID_ARG;
+    delete state;
+    return AFX_OK;
+}
+
+extern "C" afx_status afx_state_buffer(const afx_state* s, int which, int op, void** ptr, size_t* bytes) {
+    if (s == nullptr || ptr == nullptr) return AFX_ERR_INVALID_ARG;
+    size_t off = 0, sz = 0;
+    switch (which) {
+        case AFX_BUF_H: off = s->off_h; sz = s->sz_h; break;
+        case AFX_BUF_QKV: off = s->off_qkv; sz = s->sz_qkv; break;
+        case AFX_BUF_ATTN: off = s->off_attn; sz = s->sz_attn; break;
+        case AFX_BUF_HM: off = s->off_hm; sz = s->sz_hm; break;
+        case AFX_BUF_XNORM:
+            if (op != AFX_OP_QKV && op != AFX_OP_GU) return AFX_ERR_INVALID_ARG;
+            off = s->off_xnorm[op == AFX_OP_QKV ? 0 : 1]; sz = s->sz_xnorm; break;
+        case AFX_BUF_IDX:
+            if (op < 0 || op > 3) return AFX_ERR_INVALID_ARG;
+            off = s->off_idx[op]; sz = s->sz_idx[op]; break;
+        case AFX_BUF_MISS:
+            if (op < 0 || op > 3) return AFX_ERR_INVALID_ARG;
+            off = s->off_miss[op]; sz = s->sz_idx[op]; break;
+        case AFX_BUF_STATS: off = s->off_stats; sz = s->sz_stats; break;
+        default: return AFX_ERR_INVALID_ARG;
+    }
+    *ptr = s->blob + off;
+    if (bytes != nullptr) *bytes = sz;
+    return AFX_OK;
+}
+
+namespace afx {
+
+// Fills the selection part of a fused-op launch for operator input `op` of `layer`.
+static void plan_selection(const afx_model* m, const afx_state* s, int layer, int op, bool cross_layer,
+                           FusedArgs* a) {
+    const afx_model_desc& d = m->d;
+    const afx_layer_desc& L = m->layers[layer];
+    int32_t* stats = reinterpret_cast<int32_t*>(s->blob + s->off_stats);
+    int32_t* my_stats = stats + (static_cast<size_t>(layer) * 4 + op) * 4;
+    a->mode = d.select_mode;
+    a->k = L.k[op];
+    a->tau = L.tau[op];
+    a->idx_in = nullptr;
+    a->count_in = nullptr;
+    a->idx_out = reinterpret_cast<int32_t*>(s->blob + s->off_idx[op]);
+    a->count_out = my_stats + 0;
+    a->bitmap_out = nullptr;
+    a->bitmap_pred = nullptr;
+    a->miss_out = nullptr;
+    a->miss_count = nullptr;
+    a->hit_count = nullptr;
+    const int depth = d.xl_depth;
+    if (!cross_layer || depth <= 0 || d.xl_mode == AFX_XL_OFF) return;
+    const bool predictor = (layer % depth) == 0;
+    const bool predicted = layer > 0;
+    const int p = predicted ? depth * ((layer - 1) / depth) : 0;  // the layer whose set predicts this one
+    if (predicted && !predictor && d.xl_mode == AFX_XL_REUSE) {
+        a->idx_in = a->idx_out;  // the predictor's list, still in place
+        a->count_in = stats + (static_cast<size_t>(p) * 4 + op) * 4;
+        a->idx_out = nullptr;
+        return;
+    }
+    if (predicted) {
+        a->bitmap_pred = reinterpret_cast<const uint32_t*>(s->blob + s->off_pred[op][(p / depth) & 1]);
+        a->miss_out = reinterpret_cast<int32_t*>(s->blob + s->off_miss[op]);
+        a->hit_count = my_stats + 1;
+        a->miss_count = my_stats + 2;
+    }
+    if (predictor) a->bitmap_out = reinterpret_cast<uint32_t*>(s->blob + s->off_pred[op][(layer / depth) & 1]);
+}
+
+static afx_status check_step(const afx_model* m, int layer, const afx_state* s) {
+    if (m == nullptr || s == nullptr) return AFX_ERR_INVALID_ARG;
+    if (s->model != m) return AFX_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= m->d.n_layers) return AFX_ERR_INVALID_ARG;
+    return AFX_OK;
+}
+
+}  // namespace afx
+
+extern "C" afx_status afx_layer_step(afx_model* m, int layer, afx_state* s, int pos, void* stream) {
+    using namespace afx;
+    afx_status rc = check_step(m, layer, s);
+    if (rc != AFX_OK) return rc;
+    const afx_model_desc& d = m->d;
+    if (pos < 0 || pos >= d.max_seq) return AFX_ERR_INVALID_ARG;
+    const afx_layer_desc& L = m->layers[layer];
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    float* h = reinterpret_cast<float*>(s->blob + s->off_h);
+    float* qkv = reinterpret_cast<float*>(s->blob + s->off_qkv);
+    uint16_t* attn = reinterpret_cast<uint16_t*>(s->blob + s->off_attn);
+    uint16_t* hm = reinterpret_cast<uint16_t*>(s->blob + s->off_hm);
+    const int n_attn = d.n_heads * d.head_dim;
+
+    FusedArgs a = {};
+    a.T = s->T;
+    a.eps = d.rms_eps;
+    // ---- q | k | v ----
+    a.Wt = static_cast<const uint16_t*>(L.w_qkv);
+    a.ldw = m->n_qkv;
+    a.K = d.hidden;
+    a.N = m->n_qkv;
+    a.h = h;
+    a.gain = L.g_attn;
+    a.x = nullptr;
+    a.xnorm_out = reinterpret_cast<uint16_t*>(s->blob + s->off_xnorm[0]);
+    a.ep = {qkv, nullptr, m->n_qkv};
+    plan_selection(m, s, layer, AFX_OP_QKV, true, &a);
+    if ((rc = launch_fused<IN_NORM, EP_STORE>(d.dtype, a, st)) != AFX_OK) return rc;
+    // ---- rotary, cache append, dense attention ----
+    AttnArgs at = {};
+    at.qkv = qkv;
+    at.n_qkv = m->n_qkv;
+    at.q_heads = d.n_heads;
+    at.kv_heads = d.n_kv_heads;
+    at.T = s->T;
+    at.k_cache = static_cast<uint16_t*>(L.k_cache);
+    at.v_cache = static_cast<uint16_t*>(L.v_cache);
+    at.max_seq = d.max_seq;
+    at.pos = pos;
+    at.rope_cos = m->rope;
+    at.rope_sin = m->rope + static_cast<size_t>(d.max_seq) * (kHeadDim / 2);
+    at.out = attn;
+    if ((rc = launch_attention(d.dtype, at, st)) != AFX_OK) return rc;
+    // ---- o ----
+    a.Wt = static_cast<const uint16_t*>(L.w_o);
+    a.ldw = d.hidden;
+    a.K = n_attn;
+    a.N = d.hidden;
+    a.h = nullptr;
+    a.gain = nullptr;
+    a.x = attn;
+    a.xnorm_out = nullptr;
+    a.ep = {h, nullptr, d.hidden};
+    plan_selection(m, s, layer, AFX_OP_O, true, &a);
+    if ((rc = launch_fused<IN_X, EP_ACCUM>(d.dtype, a, st)) != AFX_OK) return rc;
+    // ---- gate | up, silu(gate) * up ----
+    a.Wt = static_cast<const uint16_t*>(L.w_gu);
+    a.ldw = 2 * static_cast<int64_t>(d.mlp);
+    a.K = d.hidden;
+    a.N = 2 * d.mlp;
+    a.h = h;
+    a.gain = L.g_mlp;
+    a.x = nullptr;
+    a.xnorm_out = reinterpret_cast<uint16_t*>(s->blob + s->off_xnorm[1]);
+    a.ep = {nullptr, hm, 2 * d.mlp};
+    plan_selection(m, s, layer, AFX_OP_GU, true, &a);
+    if ((rc = launch_fused<IN_NORM, EP_SILU>(d.dtype, a, st)) != AFX_OK) return rc;
+    // ---- down ----
+    a.Wt = static_cast<const uint16_t*>(L.w_down);
+    a.ldw = d.hidden;
+    a.K = d.mlp;
+    a.N = d.hidden;
+    a.h = nullptr;
+    a.gain = nullptr;
+    a.x = hm;
+    a.xnorm_out = nullptr;
+    a.ep = {h, nullptr, d.hidden};
+    plan_selection(m, s, layer, AFX_OP_DOWN, true, &a);
+    return launch_fused<IN_X, EP_ACCUM>(d.dtype, a, st);
+}
+
+extern "C" afx_status afx_mlp_block(afx_model* m, int layer, afx_state* s, const void* x, float* y,
+                                    void* stream) {
+    using namespace afx;
+    afx_status rc = check_step(m, layer, s);
+    if (rc != AFX_OK) return rc;
+    if (x == nullptr || y == nullptr) return AFX_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(x) & 1u) != 0 || !aligned16(y)) return AFX_ERR_ALIGNMENT;
+    const afx_model_desc& d = m->d;
+    const afx_layer_desc& L = m->layers[layer];
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint16_t* hm = reinterpret_cast<uint16_t*>(s->blob + s->off_hm);
+    FusedArgs a = {};
+    a.T = s->T;
+    a.eps = d.rms_eps;
+    a.Wt = static_cast<const uint16_t*>(L.w_gu);
+    a.ldw = 2 * static_cast<int64_t>(d.mlp);
+    a.K = d.hidden;
+    a.N = 2 * d.mlp;
+    a.x = static_cast<const uint16_t*>(x);
+    a.ep = {nullptr, hm, 2 * d.mlp};
+    plan_selection(m, s, layer, AFX_OP_GU, false, &a);
+    if ((rc = launch_fused<IN_X, EP_SILU>(d.dtype, a, st)) != AFX_OK) return rc;
+    a.Wt = static_cast<const uint16_t*>(L.w_down);
+    a.ldw = d.hidden;
+    a.K = d.mlp;
+    a.N = d.hidden;
+    a.x = hm;
+    a.ep = {y, nullptr, d.hidden};
+    plan_selection(m, s, layer, AFX_OP_DOWN, false, &a);
+    return launch_fused<IN_X, EP_STORE>(d.dtype, a, st);
+}

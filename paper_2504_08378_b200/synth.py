@@ -111,3 +111,48 @@ def zipf_activity_bits(seed: int, stream: int, K: int, dtype: str, alpha: float 
     mag = np.exp(score / 4.0)
     sign = np.where(g.random(K) < 0.5, -1.0, 1.0)
     return f32_to_bits((mag * sign).astype(np.float32), dtype)
+
+
+def interleave_gate_up(w_gate: np.ndarray, w_up: np.ndarray) -> np.ndarray:
+    """[K][mlp] gate and up -> [K][2*mlp] with columns in groups of 16: gate[8m..8m+8) then
+    up[8m..8m+8) (the storage layout of the fused gate/up operator; a pure re-arrangement)."""
+    K, M = w_gate.shape
+    assert w_up.shape == (K, M) and M % 8 == 0
+    out = np.empty((K, M // 8, 2, 8), w_gate.dtype)
+    out[:, :, 0, :] = w_gate.reshape(K, M // 8, 8)
+    out[:, :, 1, :] = w_up.reshape(K, M // 8, 8)
+    return out.reshape(K, 2 * M)
+
+
+def layer_weights(seed: int, layer: int, hidden: int, n_heads: int, n_kv_heads: int, mlp: int,
+                  dtype: str, head_dim: int = 128, sigma: float = 0.02, gain_jitter: float = 0.0) -> dict:
+    """Random-init weights of one Llama-shaped decoder layer (bit patterns, channel-contiguous)."""
+    base = 1000 * (layer + 1)
+    n_qkv = (n_heads + 2 * n_kv_heads) * head_dim
+    g = rng(seed, base + 7)
+    return dict(
+        w_qkv=weight(seed, base + 1, hidden, n_qkv, dtype, sigma),
+        w_o=weight(seed, base + 2, n_heads * head_dim, hidden, dtype, sigma),
+        w_gate=weight(seed, base + 3, hidden, mlp, dtype, sigma),
+        w_up=weight(seed, base + 4, hidden, mlp, dtype, sigma),
+        w_down=weight(seed, base + 5, mlp, hidden, dtype, sigma),
+        g_attn=(1.0 + gain_jitter * g.standard_normal(hidden)).astype(np.float32),
+        g_mlp=(1.0 + gain_jitter * g.standard_normal(hidden)).astype(np.float32),
+    )
+
+
+def kv_cache(seed: int, layer: int, T: int, max_seq: int, n_kv_heads: int, filled: int,
+             head_dim: int = 128):
+    """fp16 K and V caches [T][max_seq][n_kv_heads][head_dim] with `filled` past rows ~ N(0,1)."""
+    kc = np.zeros((T, max_seq, n_kv_heads, head_dim), np.uint16)
+    vc = np.zeros((T, max_seq, n_kv_heads, head_dim), np.uint16)
+    kc[:, :filled] = normal_bits(seed, 1000 * (layer + 1) + 11, (T, filled, n_kv_heads, head_dim), 1.0, "f16")
+    vc[:, :filled] = normal_bits(seed, 1000 * (layer + 1) + 12, (T, filled, n_kv_heads, head_dim), 1.0, "f16")
+    return kc, vc
+
+
+def hidden_state(seed: int, stream: int, T: int, hidden: int, scale: float = 1.0,
+                 scales_stream: int | None = None) -> np.ndarray:
+    """fp32 residual-stream input: Laplace draws times a persistent per-channel scale."""
+    a = channel_scales(seed, scales_stream, hidden) if scales_stream is not None else 1.0
+    return (laplace(seed, stream, (T, hidden), scale) * a).astype(np.float32)

@@ -41,12 +41,6 @@ def test_version_and_status_strings():
     assert afx.afx_status_string(99) == "AFX_ERR_UNKNOWN"
 
 
-def test_workspace_bytes_rejects_bad_sizes():
-    assert afx.afx_workspace_bytes(4096, 1) > 0
-    assert afx.afx_workspace_bytes(0, 1) == 0
-    assert afx.afx_workspace_bytes(4096, 9) == 0
-
-
 FAKE = 0x7F0000000000  # never dereferenced: validation fails first
 
 
@@ -74,22 +68,22 @@ def test_select_rejects_bad_arguments_on_the_host():
 
 def test_gemv_rejects_bad_arguments_on_the_host():
     ok = dict(Wt=FAKE, dtype=1, K=64, N=32, ldw=32, x=FAKE, T=1, idx=FAKE, count=FAKE, slot=None,
-              y=FAKE, acc=0, ws=FAKE)
+              y=FAKE, acc=0)
 
     def call(**kw):
         a = {**ok, **kw}
         return _status(afx.afx_sparse_gemv, a["Wt"], a["dtype"], a["K"], a["N"], a["ldw"], a["x"],
-                       a["T"], a["idx"], a["count"], a["slot"], a["y"], a["acc"], a["ws"])
+                       a["T"], a["idx"], a["count"], a["slot"], a["y"], a["acc"])
 
-    for name in ("Wt", "x", "idx", "count", "y", "ws"):
+    for name in ("Wt", "x", "idx", "count", "y"):
         assert call(**{name: None}) == 1
     assert call(K=0) == 1 and call(N=0) == 1 and call(T=0) == 1 and call(T=9) == 1
     assert call(ldw=24) == 1                       # ldw < N
     assert call(dtype=2) == 4
     assert call(N=36, ldw=40) == 2                 # N not a multiple of 8
     assert call(ldw=36) == 2                       # ldw not a multiple of 8
-    assert call(Wt=FAKE + 8) == 2 and call(y=FAKE + 4) == 2 and call(ws=FAKE + 16) == 2
-    assert call(N=8 * 40000, ldw=8 * 40000) == 3   # more column tiles than the workspace counts
+    assert call(Wt=FAKE + 8) == 2 and call(y=FAKE + 4) == 2
+    assert call(N=8 * 600000, ldw=8 * 600000) == 3  # more column tiles than a grid holds
 
 
 def test_diff_rejects_bad_arguments_on_the_host():

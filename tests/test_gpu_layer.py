@@ -1,0 +1,169 @@
+"""GPU parity for the fused decoder-layer kernels, one operator at a time: each stage's
+output is checked against the oracle run on the SAME stage input the GPU recorded."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import oracle.layer as ol
+from paper_2504_08378_b200 import afx, synth
+from paper_2504_08378_b200.model import DecoderModel
+from gpu_util import rel_err
+
+pytestmark = pytest.mark.gpu
+
+TOL = 2e-3
+OPN = ["qkv", "o", "gu", "down"]
+
+
+def bits_np(t):
+    return t.cpu().numpy().view(np.uint16)
+
+
+def ulp_close(a, b, frac_exact=0.98):
+    d = np.abs(a.astype(np.int32) - b.astype(np.int32))
+    return (d <= 1).all() and (d == 0).mean() >= frac_exact
+
+
+def make(cfg, layers_np, T, mode, xl_depth=0, xl_mode=0, max_seq=64):
+    return DecoderModel(cfg.dtype, cfg.hidden, cfg.n_heads, cfg.n_kv_heads, cfg.mlp, max_seq, layers_np, T=T,
+                        select_mode=mode, xl_depth=xl_depth, xl_mode=xl_mode)
+
+
+def oracle_weights(L, k=None, tau=None):
+    return ol.LayerWeights(L["w_qkv"], L["w_o"], L["w_gate"], L["w_up"], L["w_down"],
+                           L["g_attn"].astype(np.float64), L["g_mlp"].astype(np.float64),
+                           k=dict(zip(OPN, k or [0] * 4)), tau=dict(zip(OPN, tau or [0.0] * 4)))
+
+
+def check_layer_stages(cfg, L, lw, m, layer, h0, kc0, vc0, pos, T):
+    """Teacher-forced comparison of every stage of one layer step already run on the GPU."""
+    dt = cfg.dtype
+    Hq, Hkv, D = cfg.n_heads, cfg.n_kv_heads, cfg.head_dim
+    stats = m.stats.cpu().numpy()[layer]
+    # qkv: norm -> select -> GEMV
+    xa_gpu = bits_np(m.bits(afx.BUF_XNORM, afx.OP_QKV))
+    xa_ref = oracle.rmsnorm(h0.astype(np.float64), lw.g_attn, cfg.eps, dt)
+    assert ulp_close(xa_gpu, xa_ref)
+    idx = m.idx(afx.OP_QKV).cpu().numpy()[: stats[0][0]]
+    assert np.array_equal(idx, ol.select(xa_gpu, cfg, lw, "qkv"))
+    qkv_gpu = m.qkv.cpu().numpy()
+    qkv_ref = oracle.sparse_gemv(L["w_qkv"], dt, L["w_qkv"].shape[1], xa_gpu, idx)
+    assert rel_err(qkv_gpu, qkv_ref) <= TOL
+    # attention on the GPU's own q, k, v
+    kc, vc = kc0.copy(), vc0.copy()
+    attn_ref = ol.attention_stage(cfg, qkv_gpu.astype(np.float64), kc, vc, pos)
+    attn_gpu = bits_np(m.bits(afx.BUF_ATTN))
+    kc_gpu = bits_np(m.k_cache[layer])
+    vc_gpu = bits_np(m.v_cache[layer])
+    assert ulp_close(kc_gpu[:, pos], kc[:, pos]) and ulp_close(vc_gpu[:, pos], vc[:, pos])
+    assert np.array_equal(kc_gpu[:, :pos], kc0[:, :pos]), "past cache rows must not change"
+    a_gpu, a_ref = oracle.decode(attn_gpu, dt), oracle.decode(attn_ref, dt)
+    assert rel_err(a_gpu, a_ref) <= 2 * 2.0 ** (-8 if dt == "bf16" else -11) + 1e-3
+    # o
+    idx_o = m.idx(afx.OP_O).cpu().numpy()[: stats[1][0]]
+    assert np.array_equal(idx_o, ol.select(attn_gpu, cfg, lw, "o"))
+    h1_ref = h0.astype(np.float64) + oracle.sparse_gemv(L["w_o"], dt, cfg.hidden, attn_gpu, idx_o)
+    # gate/up
+    xm_gpu = bits_np(m.bits(afx.BUF_XNORM, afx.OP_GU))
+    assert ulp_close(xm_gpu, oracle.rmsnorm(h1_ref, lw.g_mlp, cfg.eps, dt), frac_exact=0.97)
+    idx_gu = m.idx(afx.OP_GU).cpu().numpy()[: stats[2][0]]
+    assert np.array_equal(idx_gu, ol.select(xm_gpu, cfg, lw, "gu"))
+    g = oracle.sparse_gemv(L["w_gate"], dt, cfg.mlp, xm_gpu, idx_gu)
+    u = oracle.sparse_gemv(L["w_up"], dt, cfg.mlp, xm_gpu, idx_gu)
+    hm_gpu = bits_np(m.bits(afx.BUF_HM))
+    assert ulp_close(hm_gpu, oracle.silu_mul(g, u, dt), frac_exact=0.97)
+    # down
+    idx_d = m.idx(afx.OP_DOWN).cpu().numpy()[: stats[3][0]]
+    assert np.array_equal(idx_d, ol.select(hm_gpu, cfg, lw, "down"))
+    h2_ref = h1_ref + oracle.sparse_gemv(L["w_down"], dt, cfg.hidden, hm_gpu, idx_d)
+    assert rel_err(m.h.cpu().numpy(), h2_ref) <= TOL
+    return dict(idx=[idx, idx_o, idx_gu, idx_d], stats=stats)
+
+
+@pytest.mark.parametrize("dt", ["bf16", "f16"])
+@pytest.mark.parametrize("T,mode,heads,kvh", [(1, afx.MODE_TOPK, 4, 4), (1, afx.MODE_THRESHOLD, 8, 2),
+                                              (4, afx.MODE_TOPK, 4, 4), (8, afx.MODE_TOPK, 4, 2)])
+def test_layer_step_every_stage_matches_oracle(dt, T, mode, heads, kvh):
+    hidden, mlp, max_seq, pos = heads * 128, 1384, 48, 37
+    cfg = ol.Config(dt, hidden, heads, kvh, mlp, mode=mode)
+    L = synth.layer_weights(31, 0, hidden, heads, kvh, mlp, dt, gain_jitter=0.1)
+    k = [synth.keep_count(K, 50) for K in (hidden, heads * 128, hidden, mlp)]
+    tau = [0.6, 0.02, 0.6, 0.004]
+    L["k"], L["tau"] = k, tau
+    kc0, vc0 = synth.kv_cache(31, 0, T, max_seq, kvh, pos)
+    L["k_cache"], L["v_cache"] = kc0, vc0
+    h0 = synth.hidden_state(31, 5, T, hidden, scales_stream=6)
+    m = make(cfg, [L], T, mode, max_seq=max_seq)
+    m.h.copy_(torch.from_numpy(h0).cuda())
+    m.layer_step(0, pos)
+    torch.cuda.synchronize()
+    out = check_layer_stages(cfg, L, oracle_weights(L, k, tau), m, 0, h0, kc0, vc0, pos, T)
+    if mode == afx.MODE_TOPK and T == 1:
+        assert [len(i) for i in out["idx"]] == k
+    m.close()
+
+
+@pytest.mark.parametrize("xl_mode", [afx.XL_BOOKKEEP, afx.XL_REUSE])
+def test_cross_layer_prediction_matches_oracle_free_running(xl_mode):
+    """Four layers, depth 3: free-running GPU vs free-running oracle.  Index sets are compared
+    exactly; a rare rounding flip at a top-k boundary would show up here as a set difference."""
+    dt, heads, kvh, mlp, T, max_seq, pos, depth = "bf16", 4, 4, 1024, 1, 32, 20, 3
+    hidden = heads * 128
+    cfg = ol.Config(dt, hidden, heads, kvh, mlp, mode=oracle.TOPK, xl_depth=depth, xl_mode=xl_mode)
+    layers, lws, caches = [], [], []
+    k = [synth.keep_count(K, 50) for K in (hidden, heads * 128, hidden, mlp)]
+    for l in range(4):
+        L = synth.layer_weights(41, l, hidden, heads, kvh, mlp, dt)
+        L["k"] = k
+        kc0, vc0 = synth.kv_cache(41, l, T, max_seq, kvh, pos)
+        L["k_cache"], L["v_cache"] = kc0, vc0
+        layers.append(L)
+        lws.append(oracle_weights(L, k))
+        caches.append((kc0.copy(), vc0.copy()))
+    h0 = synth.hidden_state(41, 5, T, hidden, scale=4.0, scales_stream=6)
+    m = make(cfg, layers, T, afx.MODE_TOPK, xl_depth=depth, xl_mode=xl_mode, max_seq=max_seq)
+    m.h.copy_(torch.from_numpy(h0).cuda())
+    xl = ol.CrossLayer(cfg)
+    h = h0.astype(np.float64)
+    for l in range(4):
+        m.layer_step(l, pos)
+        torch.cuda.synchronize()
+        rec = ol.decoder_layer(cfg, lws[l], h, caches[l][0], caches[l][1], pos, layer=l, xl=xl)
+        h = rec["h"]
+        stats = m.stats.cpu().numpy()[l]
+        for op, name in enumerate(OPN):
+            want = rec["idx_" + name]
+            got = m.idx(op).cpu().numpy()[: stats[op][0]]
+            assert np.array_equal(got, want), (l, name)
+            if "miss_" + name in rec:
+                assert stats[op][1] == rec["hit_" + name] and stats[op][2] == rec["miss_" + name].size
+                assert np.array_equal(m.miss(op).cpu().numpy()[: stats[op][2]], rec["miss_" + name])
+        assert rel_err(m.h.cpu().numpy(), h) <= TOL
+    m.close()
+
+
+@pytest.mark.parametrize("dt", ["f16", "bf16"])
+def test_mlp_block_threshold_sweep(dt):
+    hidden, mlp, T = 1024, 2752, 1
+    cfg = ol.Config(dt, hidden, 8, 8, mlp, mode=oracle.THRESHOLD)
+    L = synth.layer_weights(51, 0, hidden, 8, 8, mlp, dt)
+    x = synth.laplace_bits(51, 9, (T, hidden), dt)
+    for p, tau_d in ((0.0, -1.0), (0.5, 0.004), (0.9, 0.02)):
+        tau = [0.0, 0.0, synth.laplace_tau(p), tau_d]
+        L["tau"] = tau
+        m = make(cfg, [L], T, afx.MODE_THRESHOLD)
+        xd = torch.from_numpy(x.view(np.int16)).cuda()
+        y = torch.full((T, hidden), float("nan"), device="cuda")
+        m.mlp_block(0, xd, y)
+        torch.cuda.synchronize()
+        ref = ol.mlp_block(cfg, oracle_weights(L, None, tau), x)
+        stats = m.stats.cpu().numpy()[0]
+        assert np.array_equal(m.idx(afx.OP_GU).cpu().numpy()[: stats[2][0]], ref["idx_gu"])
+        hm_gpu = bits_np(m.bits(afx.BUF_HM))
+        assert ulp_close(hm_gpu, ref["hm"], frac_exact=0.97)
+        idx_d = m.idx(afx.OP_DOWN).cpu().numpy()[: stats[3][0]]
+        assert np.array_equal(idx_d, oracle.select_active(hm_gpu, dt, oracle.THRESHOLD, tau=tau_d))
+        y_ref = oracle.sparse_gemv(L["w_down"], dt, hidden, hm_gpu, idx_d)
+        assert rel_err(y.cpu().numpy(), y_ref) <= TOL
+        m.close()
