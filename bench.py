@@ -1,0 +1,381 @@
+#!/usr/bin/env python
+"""Benchmark of the active-weight decode path on B200.
+
+Workload (default): one decode token of a Llama-7B-shaped stack -- 32 layers, hidden 4096,
+32 heads x 128, MLP 11008, random-init bf16 weights, fp16 KV cache holding 2048 past
+positions -- with every q/k/v/o/gate/up/down projection evaluated on the top 50% of its
+input channels by |x| and cross-layer prediction of depth 3 kept as bookkeeping (the set
+predicted by layer l is compared with the actual sets of l+1..l+3 and the misses listed).
+A "step" is one token: 32 x afx_layer_step, captured once in a CUDA graph and replayed.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl afx|reference]
+
+prints ONE JSON line: tokens/s over all N replicas (value: inputs resident in HBM; e2e: the
+token's hidden state copied from pinned host memory and the result read back inside the
+timed region), the roofline of the dominant kernel (the fused gate/up sparse operator),
+the CPU oracle timed on a bounded sample, clocks during the timed region.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+CFG = dict(name="llama7b_decode_32L_bf16_top50_xl3", dtype="bf16", n_layers=32, hidden=4096, n_heads=32,
+           n_kv_heads=32, mlp=11008, past=2048, sparsity_percent=50, xl_depth=3, seed=3)
+ORACLE_SAMPLE_LAYERS = 2
+# dram__bytes_read.sum + dram__bytes_write.sum of one fused gate/up launch of this workload,
+# from the ncu capture summarised under profiles/ (None until captured).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def measured_peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return json.load(f), "measured"
+    except Exception:
+        return {"hbm_gbs": 6650.0}, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index, self.proc = gpu_index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            p = [c.strip() for c in line.split(",")]
+            if len(p) < 9:
+                continue
+            try:
+                sm.append(float(p[1]))
+                smax.append(float(p[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, p[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_setup(n_gpus: int):
+    """One process per GPU under torchrun; replicas only, no data-path collective."""
+    import torch
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    return world, rank, local
+
+
+def reduce_max_ms(ms: float, world: int, backend_device="cuda") -> float:
+    """Max over ranks of a duration (the slowest replica defines the job's time)."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=backend_device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def barrier(world: int):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def build_model(cfg):
+    import torch
+    from paper_2504_08378_b200 import afx, synth
+    from paper_2504_08378_b200.model import DecoderModel
+    H, M = cfg["hidden"], cfg["mlp"]
+    k = [synth.keep_count(K, cfg["sparsity_percent"]) for K in (H, cfg["n_heads"] * 128, H, M)]
+    max_seq = cfg["past"] + 8
+    layers = []
+    for l in range(cfg["n_layers"]):
+        L = synth.device_layer_weights(cfg["seed"], l, H, cfg["n_heads"], cfg["n_kv_heads"], M, cfg["dtype"])
+        L["k"] = k
+        kc = torch.zeros((1, max_seq, cfg["n_kv_heads"], 128), dtype=torch.int16, device="cuda")
+        vc = torch.zeros_like(kc)
+        kc[:, : cfg["past"]] = synth.device_normal_bits(cfg["seed"], 1000 * (l + 1) + 11,
+                                                        (1, cfg["past"], cfg["n_kv_heads"], 128), 1.0, "f16")
+        vc[:, : cfg["past"]] = synth.device_normal_bits(cfg["seed"], 1000 * (l + 1) + 12,
+                                                        (1, cfg["past"], cfg["n_kv_heads"], 128), 1.0, "f16")
+        L["k_cache"], L["v_cache"] = kc, vc
+        layers.append(L)
+    m = DecoderModel(cfg["dtype"], H, cfg["n_heads"], cfg["n_kv_heads"], M, max_seq, layers, T=1,
+                     select_mode=afx.MODE_TOPK, xl_depth=cfg["xl_depth"], xl_mode=afx.XL_BOOKKEEP)
+    return m, layers, k
+
+
+def active_bytes_per_token(cfg, k):
+    H, M = cfg["hidden"], cfg["mlp"]
+    n_qkv = (cfg["n_heads"] + 2 * cfg["n_kv_heads"]) * 128
+    per_layer = 2 * (k[0] * n_qkv + k[1] * H + k[2] * 2 * M + k[3] * H)
+    kv = 2 * 2 * (cfg["past"] + 1) * cfg["n_kv_heads"] * 128
+    return per_layer * cfg["n_layers"], kv * cfg["n_layers"]
+
+
+def run_afx(args):
+    import numpy as np
+    import torch
+    from paper_2504_08378_b200 import afx, synth
+
+    world, rank, local = dist_setup(args.gpus)
+    torch.cuda.set_device(local)
+    cfg = CFG
+    m, layers, k = build_model(cfg)
+    pos = cfg["past"]
+    h0_host = torch.from_numpy(synth.hidden_state(cfg["seed"], 5, 1, cfg["hidden"], scale=1.0,
+                                                  scales_stream=6)).pin_memory()
+    h0_dev = h0_host.cuda()
+    out_host = torch.empty_like(h0_host).pin_memory()
+    st = torch.cuda.Stream()
+
+    # one token = 32 layer steps, captured once
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(st):
+        m.h.copy_(h0_dev)
+        m.decode_step(pos, stream=st)          # warm the launch paths outside capture
+        st.synchronize()
+        with torch.cuda.graph(graph, stream=st):
+            m.h.copy_(h0_dev, non_blocking=True)
+            m.decode_step(pos, stream=st)
+    launches_per_step = 5 * cfg["n_layers"]
+
+    def timed(n_steps, e2e):
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(st):
+            ev0.record(st)
+            for _ in range(n_steps):
+                if e2e:
+                    h0_dev.copy_(h0_host, non_blocking=True)
+                graph.replay()
+                if e2e:
+                    out_host.copy_(m.h, non_blocking=True)
+                    st.synchronize()           # the caller reads the token's result
+            ev1.record(st)
+        ev1.synchronize()
+        return ev0.elapsed_time(ev1)
+
+    timed(max(args.warmup, 3), False)
+    sampler = ClockSampler(local)
+    barrier(world)
+    torch.cuda.synchronize()
+    sampler.start()
+    ms = timed(args.steps, False)
+    torch.cuda.synchronize()
+    barrier(world)
+    ms_e2e = timed(args.steps, True)
+    clocks = sampler.stop()
+    ms = reduce_max_ms(ms, world)
+    ms_e2e = reduce_max_ms(ms_e2e, world)
+
+    # ---- roofline of the dominant kernel: the fused select + sparse-GEMV operator at the
+    # gate|up shape (K 4096 -> N 22016, 45% of a token's weight bytes), launched once on each
+    # of the 32 layers' distinct weights (2.9 GB per pass, far beyond L2), timed with events
+    # on the launching stream ----
+    peaks, peak_kind = measured_peaks()
+    x_bits = synth.f32_to_bits(h0_host.numpy(), cfg["dtype"])
+    x_dev = torch.from_numpy(x_bits.view(np.int16)).cuda()
+    N_gu = 2 * cfg["mlp"]
+    y_dev = torch.empty((1, N_gu), dtype=torch.float32, device="cuda")
+
+    def gu_pass():
+        for L in layers:
+            afx.afx_select_gemv(L["w_gu"], cfg["dtype"], cfg["hidden"], N_gu, N_gu, x_dev, 1, afx.MODE_TOPK,
+                                k[2], 0.0, y_dev, 0, None, None, stream=st)
+
+    g2 = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(st):
+        gu_pass()
+        st.synchronize()
+        with torch.cuda.graph(g2, stream=st):
+            gu_pass()
+    reps = 20
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(st):
+        for _ in range(3):
+            g2.replay()
+        ev0.record(st)
+        for _ in range(reps):
+            g2.replay()
+        ev1.record(st)
+    ev1.synchronize()
+    launch_us = ev0.elapsed_time(ev1) * 1e3 / (reps * cfg["n_layers"])
+    launch_bytes = 2 * k[2] * N_gu
+    achieved = launch_bytes / (launch_us * 1e-6) / 1e9
+    roofline = {"bound": "hbm", "kernel": "fused_op_kernel (select + sparse GEMV), gate|up shape 4096->22016, k=2048",
+                "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"], "peak_kind": peak_kind, "unit": "GB/s",
+                "frac": round(achieved / peaks["hbm_gbs"], 4), "frac_of_8TBs": round(achieved / 8000.0, 4),
+                "us_per_launch": round(launch_us, 2), "algorithmic_bytes_per_launch": launch_bytes,
+                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH}
+
+    w_bytes, kv_bytes = active_bytes_per_token(cfg, k)
+    tok_s = world * args.steps / (ms * 1e-3)
+    tok_s_e2e = world * args.steps / (ms_e2e * 1e-3)
+
+    # cross-layer bookkeeping of the last token: precision |A & P| / |A| per operator input
+    m.h.copy_(h0_dev)
+    m.decode_step(pos)
+    torch.cuda.synchronize()
+    stats = m.stats.cpu().numpy().astype(np.float64)
+    pred = stats[1:]
+    precision = (pred[:, :, 1].sum(0) / np.maximum(pred[:, :, 0].sum(0), 1)).round(4).tolist()
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_baseline(cfg, layers, k, h0_host.numpy(), pos)
+
+    if rank == 0:
+        line = {
+            "metric": "decode tokens/s (batch 1)", "value": round(tok_s, 2), "unit": "tokens/s",
+            "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": round(ms / args.steps, 4), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16 weights, fp32 accumulate", "data": "synthetic",
+            "config": {"workload": cfg["name"], "layers": cfg["n_layers"], "hidden": cfg["hidden"],
+                       "mlp": cfg["mlp"], "kv_past": cfg["past"], "sparsity_percent": cfg["sparsity_percent"],
+                       "select": "top-k", "cross_layer_depth": cfg["xl_depth"], "cross_layer_mode": "bookkeeping",
+                       "l2": "6.5 GB of weights streamed per step, far larger than L2",
+                       "parallelism": f"{world} independent replica(s)"},
+            "active_weight_gbs": round(w_bytes / (ms / args.steps * 1e-3) / 1e9, 1),
+            "active_plus_kv_gbs": round((w_bytes + kv_bytes) / (ms / args.steps * 1e-3) / 1e9, 1),
+            "e2e": {"value": round(tok_s_e2e, 2), "unit": "tokens/s", "h2d_bytes_per_step": int(h0_host.numel() * 4),
+                    "d2h_bytes_per_step": int(out_host.numel() * 4)},
+            "gpu_launches": launches_per_step * args.steps,
+            "roofline": roofline, "cpu_baseline": cpu, "clocks": clocks,
+            "cross_layer_precision": dict(zip(["qkv", "o", "gate_up", "down"], precision)),
+        }
+        print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def cpu_baseline(cfg, layers, k, h0, pos):
+    """The oracle as it stands on the host cores, on the first layers of the same token."""
+    import numpy as np
+    import oracle
+    import oracle.layer as ol
+    from paper_2504_08378_b200 import synth
+    n = ORACLE_SAMPLE_LAYERS
+    ocfg = ol.Config(cfg["dtype"], cfg["hidden"], cfg["n_heads"], cfg["n_kv_heads"], cfg["mlp"], mode=oracle.TOPK)
+    lws, caches = [], []
+    for l in range(n):
+        L = layers[l]
+        host = {name: L[name].cpu().numpy().view(np.uint16) for name in ("w_qkv", "w_o", "w_gu", "w_down")}
+        wg, wu = synth.split_gate_up(host["w_gu"])
+        lws.append(ol.LayerWeights(host["w_qkv"], host["w_o"], wg, wu, host["w_down"],
+                                   np.ones(cfg["hidden"]), np.ones(cfg["hidden"]),
+                                   k=dict(zip(("qkv", "o", "gu", "down"), k))))
+        caches.append((L["k_cache"].cpu().numpy().view(np.uint16).copy(),
+                       L["v_cache"].cpu().numpy().view(np.uint16).copy()))
+    h = h0.astype(np.float64)
+    t0 = time.perf_counter()
+    for l in range(n):
+        h = ol.decoder_layer(ocfg, lws[l], h, caches[l][0], caches[l][1], pos, layer=l)["h"]
+    dt = time.perf_counter() - t0
+    return {"value": round(1.0 / (dt * cfg["n_layers"] / n), 4), "unit": "tokens/s", "cores": oracle.threads(),
+            "kind": "oracle", "sample": f"layers 0..{n - 1} of one token ({dt:.2f} s), scaled to {cfg['n_layers']} layers"}
+
+
+def run_reference(args):
+    """The oracle as the reference arm: same workload shape, bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+    import torch
+    import oracle
+    import oracle.layer as ol
+    from paper_2504_08378_b200 import synth
+    cfg = CFG
+    n = 1
+    H, M = cfg["hidden"], cfg["mlp"]
+    k = [synth.keep_count(K, cfg["sparsity_percent"]) for K in (H, cfg["n_heads"] * 128, H, M)]
+    gen = torch.Generator().manual_seed(cfg["seed"])
+
+    def w(K, N):
+        return (torch.randn(K, N, generator=gen) * 0.02).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+
+    n_qkv = (cfg["n_heads"] + 2 * cfg["n_kv_heads"]) * 128
+    lw = ol.LayerWeights(w(H, n_qkv), w(cfg["n_heads"] * 128, H), w(H, M), w(H, M), w(M, H), np.ones(H), np.ones(H),
+                         k=dict(zip(("qkv", "o", "gu", "down"), k)))
+    ocfg = ol.Config(cfg["dtype"], H, cfg["n_heads"], cfg["n_kv_heads"], M, mode=oracle.TOPK)
+    pos = cfg["past"]
+    kc, vc = synth.kv_cache(cfg["seed"], 0, 1, pos + 8, cfg["n_kv_heads"], pos)
+    h0 = synth.hidden_state(cfg["seed"], 5, 1, H, scales_stream=6).astype(np.float64)
+
+    def step():
+        ol.decoder_layer(ocfg, lw, h0, kc, vc, pos, layer=0)
+
+    for _ in range(max(1, min(args.warmup, 2))):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    ms_step = dt / args.steps * 1e3
+    val = 1.0 / (ms_step * 1e-3 * cfg["n_layers"] / n)
+    sample = f"each step = layer 0 of one token on the host, scaled to {cfg['n_layers']} layers"
+    print(json.dumps({
+        "impl": "reference", "metric": "decode tokens/s (batch 1)", "value": round(val, 4), "unit": "tokens/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms_step, 3),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64 (oracle)",
+        "data": "synthetic", "config": {"workload": cfg["name"], "sample": sample},
+        "cpu_baseline": {"value": round(val, 4), "unit": "tokens/s", "cores": oracle.threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": round(val, 4), "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="afx", choices=["afx", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_afx(args)
+
+
+if __name__ == "__main__":
+    main()

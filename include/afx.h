@@ -105,6 +105,20 @@ afx_status afx_sparse_gemv(const void* Wt, int dtype, int K, int N, int64_t ldw,
                            int T, const int32_t* idx, const int32_t* count, const int32_t* slot,
                            float* y, int accumulate, void* stream);
 
+/*
+ * Selection and sparse GEMV in ONE kernel (the T and C operations of Sec. 4 back to back):
+ * the result equals afx_select_active followed by afx_sparse_gemv on the same arguments,
+ * without the list's round trip through global memory between two launches.
+ *
+ *   Wt, x, y, accumulate   as for afx_sparse_gemv;  mode, k, tau  as for afx_select_active.
+ *   idx_out   DEVICE int32[K] or NULL: receives the active list.
+ *   count_out DEVICE int32[1] or NULL: receives its length.
+ * K * T * 2 bytes of x are read by every thread block (they stay in L2).
+ */
+afx_status afx_select_gemv(const void* Wt, int dtype, int K, int N, int64_t ldw, const void* x, int T,
+                           int mode, int k, float tau, float* y, int accumulate, int32_t* idx_out,
+                           int32_t* count_out, void* stream);
+
 /* ------------------------------------------------------------------------------------------
  * Decoder layers: every linear operator of a Llama-shaped layer run as ONE kernel that
  * normalises (where the layer does), selects the active channels of its own input and

@@ -65,6 +65,8 @@ def lib() -> ctypes.CDLL:
                                       c_void_p, c_void_p]
         L.afx_sparse_gemv.argtypes = [c_void_p, c_int, c_int, c_int, c_int64, c_void_p, c_int,
                                       c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p]
+        L.afx_select_gemv.argtypes = [c_void_p, c_int, c_int, c_int, c_int64, c_void_p, c_int, c_int, c_int,
+                                      c_float, c_void_p, c_int, c_void_p, c_void_p, c_void_p]
         L.afx_model_create.argtypes = [ctypes.POINTER(ModelDesc), ctypes.POINTER(LayerDesc),
                                        ctypes.POINTER(c_void_p)]
         L.afx_model_destroy.argtypes = [c_void_p]
@@ -135,6 +137,14 @@ def afx_sparse_gemv(Wt, dtype, K: int, N: int, ldw: int, x, T: int, idx, count, 
     _check("afx_sparse_gemv",
            lib().afx_sparse_gemv(_ptr(Wt), _dt(dtype), int(K), int(N), int(ldw), _ptr(x), int(T),
                                  _ptr(idx), _ptr(count), _ptr(slot), _ptr(y), int(accumulate),
+                                 _stream(stream)))
+
+
+def afx_select_gemv(Wt, dtype, K: int, N: int, ldw: int, x, T: int, mode: int, k: int, tau: float, y,
+                    accumulate: int, idx_out=None, count_out=None, stream=None):
+    _check("afx_select_gemv",
+           lib().afx_select_gemv(_ptr(Wt), _dt(dtype), int(K), int(N), int(ldw), _ptr(x), int(T), int(mode),
+                                 int(k), float(tau), _ptr(y), int(accumulate), _ptr(idx_out), _ptr(count_out),
                                  _stream(stream)))
 
 

@@ -425,3 +425,35 @@ extern "C" afx_status afx_mlp_block(afx_model* m, int layer, afx_state* s, const
     plan_selection(m, s, layer, AFX_OP_DOWN, false, &a);
     return launch_fused<IN_X, EP_STORE>(d.dtype, a, st);
 }
+
+extern "C" afx_status afx_select_gemv(const void* Wt, int dtype, int K, int N, int64_t ldw, const void* x, int T,
+                                      int mode, int k, float tau, float* y, int accumulate, int32_t* idx_out,
+                                      int32_t* count_out, void* stream) {
+    using namespace afx;
+    if (Wt == nullptr || x == nullptr || y == nullptr) return AFX_ERR_INVALID_ARG;
+    if (K <= 0 || K > (1 << 20) || N <= 0 || T < 1 || T > AFX_MAX_T || ldw < N) return AFX_ERR_INVALID_ARG;
+    if (dtype != AFX_F16 && dtype != AFX_BF16) return AFX_ERR_UNSUPPORTED;
+    if (mode != AFX_MODE_TOPK && mode != AFX_MODE_THRESHOLD) return AFX_ERR_UNSUPPORTED;
+    if (mode == AFX_MODE_TOPK && (k < 0 || k > K)) return AFX_ERR_INVALID_ARG;
+    if (mode == AFX_MODE_THRESHOLD && tau != tau) return AFX_ERR_INVALID_ARG;
+    if ((N & 7) != 0 || (ldw & 7) != 0 || !aligned16(Wt) || !aligned16(y) ||
+        (reinterpret_cast<uintptr_t>(x) & 1u) != 0 || (reinterpret_cast<uintptr_t>(idx_out) & 3u) != 0 ||
+        (reinterpret_cast<uintptr_t>(count_out) & 3u) != 0)
+        return AFX_ERR_ALIGNMENT;
+    if ((N + 63) / 64 > 65535) return AFX_ERR_CAPACITY;
+    FusedArgs a = {};
+    a.Wt = static_cast<const uint16_t*>(Wt);
+    a.ldw = ldw;
+    a.K = K;
+    a.N = N;
+    a.T = T;
+    a.x = static_cast<const uint16_t*>(x);
+    a.mode = mode;
+    a.k = k;
+    a.tau = tau;
+    a.ep = {y, nullptr, N};
+    a.idx_out = idx_out;
+    a.count_out = count_out;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return accumulate ? launch_fused<IN_X, EP_ACCUM>(dtype, a, st) : launch_fused<IN_X, EP_STORE>(dtype, a, st);
+}

@@ -14,7 +14,9 @@ from . import afx, synth
 _TORCH_16 = {"f16": torch.float16, "bf16": torch.bfloat16}
 
 
-def to_device_bits(a: np.ndarray) -> torch.Tensor:
+def to_device_bits(a) -> torch.Tensor:
+    if isinstance(a, torch.Tensor):
+        return a.cuda().contiguous()
     a = np.ascontiguousarray(a)
     if a.dtype == np.uint16:
         return torch.from_numpy(a.view(np.int16)).cuda()
@@ -43,10 +45,9 @@ class DecoderModel:
             d = afx.LayerDesc()
             w_gu = L["w_gu"] if "w_gu" in L else synth.interleave_gate_up(L["w_gate"], L["w_up"])
             tens = dict(w_qkv=to_device_bits(L["w_qkv"]), w_o=to_device_bits(L["w_o"]),
-                        w_gu=to_device_bits(w_gu) if isinstance(w_gu, np.ndarray) else w_gu,
+                        w_gu=to_device_bits(w_gu),
                         w_down=to_device_bits(L["w_down"]),
-                        g_attn=to_device_bits(np.asarray(L["g_attn"], np.float32)),
-                        g_mlp=to_device_bits(np.asarray(L["g_mlp"], np.float32)))
+                        g_attn=to_device_bits(L["g_attn"]).float(), g_mlp=to_device_bits(L["g_mlp"]).float())
             if "k_cache" in L:
                 kc, vc = to_device_bits(L["k_cache"]), to_device_bits(L["v_cache"])
             else:

@@ -156,3 +156,48 @@ def hidden_state(seed: int, stream: int, T: int, hidden: int, scale: float = 1.0
     """fp32 residual-stream input: Laplace draws times a persistent per-channel scale."""
     a = channel_scales(seed, scales_stream, hidden) if scales_stream is not None else 1.0
     return (laplace(seed, stream, (T, hidden), scale) * a).astype(np.float32)
+
+
+# ---- device-side draws (bench-scale tensors: 13+ GB are drawn on the GPU in a second) ----
+
+def device_normal_bits(seed: int, stream: int, shape, sigma: float, dtype: str):
+    """N(0, sigma^2) rounded to dtype, drawn with torch's seeded CUDA generator.
+    Returns an int16 CUDA tensor of bit patterns.  Input generation only."""
+    import torch
+    g = torch.Generator(device="cuda")
+    g.manual_seed((int(seed) * 1000003 + int(stream)) & (2**63 - 1))
+    tdt = torch.float16 if dtype == "f16" else torch.bfloat16
+    n = 1
+    for s in shape:
+        n *= int(s)
+    out = torch.empty(n, dtype=tdt, device="cuda")
+    chunk = 1 << 26
+    for o in range(0, n, chunk):
+        m = min(chunk, n - o)
+        out[o:o + m] = (torch.randn(m, generator=g, device="cuda", dtype=torch.float32) * sigma).to(tdt)
+    return out.view(torch.int16).view(*shape)
+
+
+def device_layer_weights(seed: int, layer: int, hidden: int, n_heads: int, n_kv_heads: int, mlp: int,
+                         dtype: str, head_dim: int = 128, sigma: float = 0.02) -> dict:
+    """Device-resident random-init layer (w_gu already in the interleaved gate/up layout:
+    with i.i.d. entries any fixed column arrangement has the same distribution)."""
+    import torch
+    base = 1000 * (layer + 1)
+    n_qkv = (n_heads + 2 * n_kv_heads) * head_dim
+    return dict(
+        w_qkv=device_normal_bits(seed, base + 1, (hidden, n_qkv), sigma, dtype),
+        w_o=device_normal_bits(seed, base + 2, (n_heads * head_dim, hidden), sigma, dtype),
+        w_gu=device_normal_bits(seed, base + 3, (hidden, 2 * mlp), sigma, dtype),
+        w_down=device_normal_bits(seed, base + 5, (mlp, hidden), sigma, dtype),
+        g_attn=torch.ones(hidden, dtype=torch.float32, device="cuda"),
+        g_mlp=torch.ones(hidden, dtype=torch.float32, device="cuda"),
+    )
+
+
+def split_gate_up(w_gu: np.ndarray):
+    """Inverse of interleave_gate_up: [K][2*mlp] -> (gate [K][mlp], up [K][mlp])."""
+    K, N2 = w_gu.shape
+    v = w_gu.reshape(K, N2 // 16, 2, 8)
+    return (np.ascontiguousarray(v[:, :, 0, :]).reshape(K, N2 // 2),
+            np.ascontiguousarray(v[:, :, 1, :]).reshape(K, N2 // 2))

@@ -136,3 +136,23 @@ def test_integer_weights_give_exact_results():
         assert np.array_equal(y[0].astype(np.float64),
                               oracle.sparse_gemv(synth.f32_to_bits(W, dt), dt, N,
                                                  synth.f32_to_bits(xv, dt), idx)[0])
+
+
+@pytest.mark.parametrize("dt", ["f16", "bf16"])
+@pytest.mark.parametrize("K,N,T", [(512, 1376, 1), (4096, 2048 + 40, 1), (1000, 4096, 3), (2048, 11008, 1)])
+def test_select_gemv_equals_select_then_gemv(dt, K, N, T):
+    """The one-kernel form: list bit-exact, y within tolerance of the oracle."""
+    Wt = synth.weight(211, K + N, K, N, dt)
+    x = synth.laplace_bits(212, K, (T, K), dt)
+    W, xd = dev_bits(Wt), dev_bits(x)
+    for mode, kw in ((afx.MODE_TOPK, dict(k=synth.keep_count(K, 50))), (afx.MODE_TOPK, dict(k=0)),
+                     (afx.MODE_THRESHOLD, dict(tau=synth.laplace_tau(0.7))), (afx.MODE_THRESHOLD, dict(tau=-1.0))):
+        idx_d = torch.full((K,), -3, dtype=torch.int32, device="cuda")
+        cnt_d = torch.full((1,), -3, dtype=torch.int32, device="cuda")
+        y = torch.full((T, N), float("nan"), dtype=torch.float32, device="cuda")
+        afx.afx_select_gemv(W, dt, K, N, N, xd, T, mode, kw.get("k", 0), kw.get("tau", 0.0), y, 0, idx_d, cnt_d)
+        torch.cuda.synchronize()
+        want = oracle.select_active(x, dt, mode, **kw)
+        n = int(cnt_d.item())
+        assert n == want.size and np.array_equal(idx_d.cpu().numpy()[:n], want)
+        assert rel_err(y.cpu().numpy(), oracle.sparse_gemv(Wt, dt, N, x, want)) <= TOL
