@@ -3,7 +3,7 @@
 //
 // grid = (S, kv_heads, T), cluster = (S,1,1): the S blocks of a cluster split the L = pos+1
 // cached positions of one (token, kv head) and meet their (max, sum, weighted V) partials
-// through distributed shared memory.  The block owning the last position first rotates and
+// through distributed shared memory (softmax in base 2: exp(s) = 2^(s * log2 e)).  The block owning the last position first rotates and
 // stores the current token's k and v into the cache.  head_dim is fixed at 128.
 #pragma once
 
@@ -17,10 +17,10 @@ namespace cg = cooperative_groups;
 
 constexpr int kAttnThreads = 256;
 constexpr int kAttnWarps = kAttnThreads / 32;
+constexpr int kAttnWorkers = 2 * kAttnWarps;  // half warps: each walks its own positions
 constexpr int kHeadDim = 128;
-constexpr int kAttnKeyBlock = 256;
 constexpr int kAttnMaxRep = 8;  // query heads per kv head
-constexpr int kAttnUnroll = 4;  // cache rows in flight per half warp
+constexpr int kAttnUnroll = 4;  // cache rows (K and V each) in flight per half warp
 
 struct AttnArgs {
     const float* qkv;  // [T][n_qkv] fp32: q heads | k heads | v heads
@@ -34,11 +34,11 @@ struct AttnArgs {
 };
 
 struct AttnSmem {
-    float q[kAttnMaxRep][kHeadDim];
-    float score[kAttnMaxRep][kAttnKeyBlock];
-    __align__(16) float red[2 * kAttnWarps][kHeadDim];
-    float m_new[kAttnMaxRep];
-    float part_m[kAttnMaxRep];
+    __align__(16) float q[kAttnMaxRep][kHeadDim];     // rotated queries times scale * log2(e)
+    __align__(16) float red[kAttnWorkers][kHeadDim];  // one query head's partial outputs
+    float red_m[kAttnWorkers];
+    float red_l[kAttnWorkers];
+    float part_m[kAttnMaxRep];  // this block's partials, read by the cluster
     float part_l[kAttnMaxRep];
     float part_acc[kAttnMaxRep][kHeadDim];
 };
@@ -53,7 +53,18 @@ __device__ __forceinline__ void unpack8_f16(const uint4& raw, float (&w)[8]) {
     }
 }
 
-template <int DT>
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// One pass over the cache: every half warp keeps a running (max, sum, weighted V) per query
+// head for the positions it visits (16 lanes x 8 dims = one 128-wide row per load), K and V
+// rows of kAttnUnroll positions are requested together so that 2 * kAttnUnroll 16-byte loads
+// per lane are in flight; the half warps of a block meet in shared memory, the blocks of a
+// cluster through distributed shared memory, both in a fixed order.
+template <int DT, int REP>
 __device__ __forceinline__ void attention_block(const AttnArgs& a, AttnSmem* sm) {
     cg::cluster_group cluster = cg::this_cluster();
     const int S = static_cast<int>(cluster.num_blocks());
@@ -61,11 +72,12 @@ __device__ __forceinline__ void attention_block(const AttnArgs& a, AttnSmem* sm)
     const int hk = blockIdx.y, t = blockIdx.z;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int half = lane >> 4, l16 = lane & 15;
+    const int worker = 2 * warp + half;
     const int rep = a.q_heads / a.kv_heads;
     const int L = a.pos + 1;
     const int l_lo = static_cast<int>(static_cast<int64_t>(rank) * L / S);
     const int l_hi = static_cast<int>(static_cast<int64_t>(rank + 1) * L / S);
-    const float scale = rsqrtf(static_cast<float>(kHeadDim));
+    const float qscale = rsqrtf(static_cast<float>(kHeadDim)) * 1.4426950408889634f;
     const uint32_t half_mask = 0xFFFFu << (16 * half);  // the two halves of a warp work on different keys
 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -77,14 +89,15 @@ __device__ __forceinline__ void attention_block(const AttnArgs& a, AttnSmem* sm)
     uint16_t* kc = a.k_cache + static_cast<size_t>(t) * a.max_seq * a.kv_heads * kHeadDim;
     uint16_t* vc = a.v_cache + static_cast<size_t>(t) * a.max_seq * a.kv_heads * kHeadDim;
     const size_t row_stride = static_cast<size_t>(a.kv_heads) * kHeadDim;
+    const size_t head_off = static_cast<size_t>(hk) * kHeadDim + l16 * 8;
 
-    // rotated queries of this kv head's group
+    // rotated, pre-scaled queries of this kv head's group
     for (int e = tid; e < rep * (kHeadDim / 2); e += kAttnThreads) {
         const int r = e / (kHeadDim / 2), i = e - r * (kHeadDim / 2);
         const float* qh = row + static_cast<size_t>(hk * rep + r) * kHeadDim;
         const float x0 = qh[2 * i], x1 = qh[2 * i + 1];
-        sm->q[r][2 * i] = x0 * cs[i] - x1 * sn[i];
-        sm->q[r][2 * i + 1] = x0 * sn[i] + x1 * cs[i];
+        sm->q[r][2 * i] = (x0 * cs[i] - x1 * sn[i]) * qscale;
+        sm->q[r][2 * i + 1] = (x0 * sn[i] + x1 * cs[i]) * qscale;
     }
     // the block that owns the newest position appends the current k, v (fp16) first
     if (l_hi == L && l_lo < l_hi) {
@@ -103,121 +116,110 @@ __device__ __forceinline__ void attention_block(const AttnArgs& a, AttnSmem* sm)
     }
     __syncthreads();
 
-    float m_run[kAttnMaxRep], l_run[kAttnMaxRep], acc[kAttnMaxRep][8];
+    float m_run[REP], l_run[REP], acc[REP][8];
 #pragma unroll
-    for (int r = 0; r < kAttnMaxRep; ++r) {
+    for (int r = 0; r < REP; ++r) {
         m_run[r] = -INFINITY;
         l_run[r] = 0.0f;
 #pragma unroll
         for (int j = 0; j < 8; ++j) acc[r][j] = 0.0f;
     }
 
-    for (int b0 = l_lo; b0 < l_hi; b0 += kAttnKeyBlock) {
-        const int nb = min(kAttnKeyBlock, l_hi - b0);
-        // pass 1: scores of the block's keys (half a warp per key, kAttnUnroll keys in flight)
-        for (int i0 = 2 * warp + half; i0 < nb; i0 += 2 * kAttnWarps * kAttnUnroll) {
-            uint4 raw[kAttnUnroll];
+    constexpr int U = kAttnUnroll;
+    for (int p0 = l_lo + worker; p0 < l_hi; p0 += kAttnWorkers * U) {
+        uint4 kraw[U], vraw[U];
 #pragma unroll
-            for (int u = 0; u < kAttnUnroll; ++u) {
-                const int i = i0 + u * 2 * kAttnWarps;
-                if (i < nb)
-                    raw[u] = *reinterpret_cast<const uint4*>(kc + static_cast<size_t>(b0 + i) * row_stride +
-                                                             static_cast<size_t>(hk) * kHeadDim + l16 * 8);
+        for (int u = 0; u < U; ++u) {
+            const int p = p0 + u * kAttnWorkers;
+            if (p < l_hi) {
+                kraw[u] = *reinterpret_cast<const uint4*>(kc + static_cast<size_t>(p) * row_stride + head_off);
+                vraw[u] = *reinterpret_cast<const uint4*>(vc + static_cast<size_t>(p) * row_stride + head_off);
             }
+        }
+        float sc[REP][U];
 #pragma unroll
-            for (int u = 0; u < kAttnUnroll; ++u) {
-                const int i = i0 + u * 2 * kAttnWarps;
-                if (i < nb) {
-                    float kv[8];
-                    unpack8_f16(raw[u], kv);
+        for (int r = 0; r < REP; ++r) {
+            if (r < rep) {
+                const float4 qa = *reinterpret_cast<const float4*>(&sm->q[r][l16 * 8]);
+                const float4 qb = *reinterpret_cast<const float4*>(&sm->q[r][l16 * 8 + 4]);
 #pragma unroll
-                    for (int r = 0; r < kAttnMaxRep; ++r) {
-                        if (r < rep) {
-                            float d = 0.0f;
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) d = fmaf(sm->q[r][l16 * 8 + j], kv[j], d);
-                            d += __shfl_xor_sync(half_mask, d, 8);
-                            d += __shfl_xor_sync(half_mask, d, 4);
-                            d += __shfl_xor_sync(half_mask, d, 2);
-                            d += __shfl_xor_sync(half_mask, d, 1);
-                            if (l16 == 0) sm->score[r][i] = d * scale;
-                        }
+                for (int u = 0; u < U; ++u) {
+                    float d = -INFINITY;
+                    if (p0 + u * kAttnWorkers < l_hi) {  // uniform over the half warp
+                        float kv[8];
+                        unpack8_f16(kraw[u], kv);
+                        d = qa.x * kv[0];
+                        d = fmaf(qa.y, kv[1], d);
+                        d = fmaf(qa.z, kv[2], d);
+                        d = fmaf(qa.w, kv[3], d);
+                        d = fmaf(qb.x, kv[4], d);
+                        d = fmaf(qb.y, kv[5], d);
+                        d = fmaf(qb.z, kv[6], d);
+                        d = fmaf(qb.w, kv[7], d);
+                        d += __shfl_xor_sync(half_mask, d, 8);
+                        d += __shfl_xor_sync(half_mask, d, 4);
+                        d += __shfl_xor_sync(half_mask, d, 2);
+                        d += __shfl_xor_sync(half_mask, d, 1);
                     }
+                    sc[r][u] = d;
                 }
             }
         }
-        __syncthreads();
-        // new running maximum per query head (warp r handles head r)
-        if (warp < rep) {
-            float mx = -INFINITY;
-            for (int i = lane; i < nb; i += 32) mx = fmaxf(mx, sm->score[warp][i]);
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
-            if (lane == 0) sm->m_new[warp] = mx;
-        }
-        __syncthreads();
-        // pass 2: weights and weighted values
-#pragma unroll
-        for (int r = 0; r < kAttnMaxRep; ++r) {
+        for (int r = 0; r < REP; ++r) {
             if (r < rep) {
-                const float mn = fmaxf(m_run[r], sm->m_new[r]);
-                const float f = expf(m_run[r] - mn);  // exp(-inf) = 0 on the first block
+                float mn = m_run[r];
+#pragma unroll
+                for (int u = 0; u < U; ++u) mn = fmaxf(mn, sc[r][u]);
+                const float f = fast_exp2(m_run[r] - mn);  // 0 on the first visit (m_run = -inf)
+                m_run[r] = mn;
                 l_run[r] *= f;
 #pragma unroll
                 for (int j = 0; j < 8; ++j) acc[r][j] *= f;
-                m_run[r] = mn;
-            }
-        }
-        for (int i0 = 2 * warp + half; i0 < nb; i0 += 2 * kAttnWarps * kAttnUnroll) {
-            uint4 raw[kAttnUnroll];
 #pragma unroll
-            for (int u = 0; u < kAttnUnroll; ++u) {
-                const int i = i0 + u * 2 * kAttnWarps;
-                if (i < nb)
-                    raw[u] = *reinterpret_cast<const uint4*>(vc + static_cast<size_t>(b0 + i) * row_stride +
-                                                             static_cast<size_t>(hk) * kHeadDim + l16 * 8);
-            }
+                for (int u = 0; u < U; ++u) {
+                    if (p0 + u * kAttnWorkers < l_hi) {
+                        const float pw = fast_exp2(sc[r][u] - mn);
+                        l_run[r] += pw;
+                        float vv[8];
+                        unpack8_f16(vraw[u], vv);
 #pragma unroll
-            for (int u = 0; u < kAttnUnroll; ++u) {
-                const int i = i0 + u * 2 * kAttnWarps;
-                if (i < nb) {
-                    float vv[8];
-                    unpack8_f16(raw[u], vv);
-#pragma unroll
-                    for (int r = 0; r < kAttnMaxRep; ++r) {
-                        if (r < rep) {
-                            const float p = expf(sm->score[r][i] - m_run[r]);
-                            l_run[r] += p;
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) acc[r][j] = fmaf(p, vv[j], acc[r][j]);
-                        }
+                        for (int j = 0; j < 8; ++j) acc[r][j] = fmaf(pw, vv[j], acc[r][j]);
                     }
                 }
             }
         }
-        __syncthreads();
     }
 
-    // meet the 16 key groups of the block (fixed order), one query head at a time
+    // meet the half warps of the block (fixed order), one query head at a time
 #pragma unroll
-    for (int r = 0; r < kAttnMaxRep; ++r) {
+    for (int r = 0; r < REP; ++r) {
         if (r < rep) {
-            float4* dst = reinterpret_cast<float4*>(&sm->red[2 * warp + half][l16 * 8]);
+            float4* dst = reinterpret_cast<float4*>(&sm->red[worker][l16 * 8]);
             dst[0] = make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
             dst[1] = make_float4(acc[r][4], acc[r][5], acc[r][6], acc[r][7]);
-            if (l16 == 0) sm->score[0][2 * warp + half] = l_run[r];  // score[] is free now
+            if (l16 == 0) {
+                sm->red_m[worker] = m_run[r];
+                sm->red_l[worker] = l_run[r];
+            }
             __syncthreads();
-            if (tid < kHeadDim) {
+            if (tid <= kHeadDim) {
+                float M = -INFINITY;
+#pragma unroll
+                for (int g = 0; g < kAttnWorkers; ++g) M = fmaxf(M, sm->red_m[g]);
                 float s = 0.0f;
 #pragma unroll
-                for (int g = 0; g < 2 * kAttnWarps; ++g) s += sm->red[g][tid];
-                sm->part_acc[r][tid] = s;
-            } else if (tid == kHeadDim) {
-                float s = 0.0f;
-#pragma unroll
-                for (int g = 0; g < 2 * kAttnWarps; ++g) s += sm->score[0][g];
-                sm->part_l[r] = s;
-                sm->part_m[r] = m_run[r];  // identical in every thread of the block
+                for (int g = 0; g < kAttnWorkers; ++g) {
+                    // a half warp that saw no position has m = -inf, l = 0, acc = 0
+                    const float w = sm->red_m[g] == -INFINITY ? 0.0f : fast_exp2(sm->red_m[g] - M);
+                    s = fmaf(w, tid < kHeadDim ? sm->red[g][tid] : sm->red_l[g], s);
+                }
+                if (tid < kHeadDim) {
+                    sm->part_acc[r][tid] = s;
+                } else {
+                    sm->part_l[r] = s;
+                    sm->part_m[r] = M;
+                }
             }
             __syncthreads();
         }
@@ -229,7 +231,8 @@ __device__ __forceinline__ void attention_block(const AttnArgs& a, AttnSmem* sm)
         for (int q = 0; q < S; ++q) M = fmaxf(M, cluster.map_shared_rank(&sm->part_m[0], q)[r]);
         float num = 0.0f, den = 0.0f;
         for (int q = 0; q < S; ++q) {
-            const float w = expf(cluster.map_shared_rank(&sm->part_m[0], q)[r] - M);
+            const float mq = cluster.map_shared_rank(&sm->part_m[0], q)[r];
+            const float w = mq == -INFINITY ? 0.0f : fast_exp2(mq - M);
             num = fmaf(w, cluster.map_shared_rank(&sm->part_acc[0][0], q)[r * kHeadDim + d], num);
             den = fmaf(w, cluster.map_shared_rank(&sm->part_l[0], q)[r], den);
         }

@@ -7,6 +7,21 @@
 
 #include "afx.h"
 
+// Stage marks for kernel timing studies: compiled out unless AFX_TRACE is defined, in which
+// case thread 0 of every block stores the SM clock of mark i into afx_trace_buf.
+#ifdef AFX_TRACE
+extern __device__ long long afx_trace_buf[];
+#define AFX_MARK(i)                                                                              \
+    do {                                                                                         \
+        if (threadIdx.x == 0)                                                                    \
+            afx_trace_buf[((blockIdx.y * gridDim.x + blockIdx.x) % 512) * 16 + (i)] = clock64(); \
+    } while (0)
+#else
+#define AFX_MARK(i) \
+    do {            \
+    } while (0)
+#endif
+
 namespace afx {
 
 constexpr int kWarp = 32;

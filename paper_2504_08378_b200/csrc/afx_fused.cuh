@@ -38,17 +38,24 @@ struct FusedArgs {
     int32_t* hit_count;           // |A & P|
 };
 
-// Dynamic shared memory: [T*K 16-bit inputs (IN_NORM only)] [ceil(K/32) flag words].
+// Dynamic shared memory: [16-bit inputs: T tokens (IN_NORM) or one token (IN_X), each padded
+// to a multiple of 8 elements] [ceil(K/32) flag words, padded to 16 bytes] [work area: the key
+// histogram during the selection, then the GEMV staging and reduction buffers].
+__host__ __device__ inline size_t fused_input_smem(int in_kind, int K, int T) {
+    const size_t Kp = (static_cast<size_t>(K) + 7) / 8 * 8;
+    return (in_kind == IN_NORM ? static_cast<size_t>(T) : 1) * Kp * 2;
+}
+__host__ __device__ inline size_t fused_flag_smem(int K) {
+    return (static_cast<size_t>((K + 31) / 32) * 4 + 15) / 16 * 16;
+}
 __host__ __device__ inline size_t fused_dyn_smem(int in_kind, int K, int T) {
-    size_t b = static_cast<size_t>((K + 31) / 32) * 4;
-    if (in_kind == IN_NORM) b += (static_cast<size_t>(T) * K * 2 + 15) / 16 * 16;
-    return b;
+    return fused_input_smem(in_kind, K, T) + fused_flag_smem(K) + kKeyHistBytes;
 }
 
 template <int DT, int TMAX, int PW, int CAP, int IN, int EP>
-__device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char* dyn,
-                                               GemvSmem<TMAX, CAP>* sm, SelectScratch* sel) {
+__device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char* dyn, SelectScratch* sel) {
     constexpr int LPC = PW / 8;
+    static_assert(sizeof(GemvSmem<TMAX, CAP>) <= kKeyHistBytes, "work area too small");
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int warp = tid >> 5;
@@ -57,63 +64,109 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
     const bool scribe = (blockIdx.x == 0 && blockIdx.y == 0);  // writes the side outputs
     const int nwords = (K + 31) >> 5;
 
+    const int Kp = (K + 7) & ~7;
     uint16_t* xs = reinterpret_cast<uint16_t*>(dyn);
-    uint32_t* flags = reinterpret_cast<uint32_t*>(
-        dyn + (IN == IN_NORM ? (static_cast<size_t>(T) * K * 2 + 15) / 16 * 16 : 0));
+    uint32_t* flags = reinterpret_cast<uint32_t*>(dyn + fused_input_smem(IN, K, T));
+    unsigned char* work = dyn + fused_input_smem(IN, K, T) + fused_flag_smem(K);
+    uint32_t* hist = reinterpret_cast<uint32_t*>(work);
+    GemvSmem<TMAX, CAP>* sm = reinterpret_cast<GemvSmem<TMAX, CAP>*>(work);
+    float* red16 = reinterpret_cast<float*>(sel->hist);  // block reduction of the norm
+
+    const bool own = (a.idx_in == nullptr);
+    const bool topk = own && a.mode == AFX_MODE_TOPK && a.k > 0 && a.k < K;
+    AFX_MARK(0);
+    if (topk) block_clear_key_hist(hist);  // does not depend on the previous kernel
 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    AFX_MARK(1);
 
     // ---- input stage --------------------------------------------------------------------
-    const uint16_t* xin = a.x;
     if (IN == IN_NORM) {
+        // x = round(h / rms(h) * gain), every block for itself (K % 8 == 0, 16-byte aligned rows)
+        constexpr int NH = 4;  // float4 pieces of h a thread keeps between the two passes
+        const int nq = K >> 2;
         for (int t = 0; t < T; ++t) {
-            const float* ht = a.h + static_cast<size_t>(t) * K;
+            const float4* ht = reinterpret_cast<const float4*>(a.h + static_cast<size_t>(t) * K);
+            float4 hv[NH];
             float ss = 0.0f;
-            for (int j = tid; j < K; j += kGemvThreads) {
-                const float v = ht[j];
-                ss = fmaf(v, v, ss);
+#pragma unroll
+            for (int i = 0; i < NH; ++i) {
+                const int c = tid + i * kGemvThreads;
+                hv[i] = c < nq ? ht[c] : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                ss = fmaf(hv[i].x, hv[i].x, ss);
+                ss = fmaf(hv[i].y, hv[i].y, ss);
+                ss = fmaf(hv[i].z, hv[i].z, ss);
+                ss = fmaf(hv[i].w, hv[i].w, ss);
+            }
+            for (int c = tid + NH * kGemvThreads; c < nq; c += kGemvThreads) {
+                const float4 v = ht[c];
+                ss = fmaf(v.x, v.x, ss);
+                ss = fmaf(v.y, v.y, ss);
+                ss = fmaf(v.z, v.z, ss);
+                ss = fmaf(v.w, v.w, ss);
             }
             ss = warp_sum(ss);
             __syncthreads();
-            if (lane == 0) sm->red[0][warp] = ss;
+            if (lane == 0) red16[warp] = ss;
             __syncthreads();
             float tot = 0.0f;
 #pragma unroll
-            for (int w = 0; w < kGemvWarps; ++w) tot += sm->red[0][w];
+            for (int w = 0; w < kGemvWarps; ++w) tot += red16[w];
             const float inv = 1.0f / sqrtf(tot / static_cast<float>(K) + a.eps);
-            for (int j = tid; j < K; j += kGemvThreads) {
-                const uint16_t b = float_to_bits<DT>(ht[j] * inv * a.gain[j]);
-                xs[static_cast<size_t>(t) * K + j] = b;
-                if (scribe && a.xnorm_out != nullptr) a.xnorm_out[static_cast<size_t>(t) * K + j] = b;
+            const float4* gq = reinterpret_cast<const float4*>(a.gain);
+            auto emit = [&](int c, const float4& v) {
+                const float4 g = gq[c];
+                const uint32_t lo = static_cast<uint32_t>(float_to_bits<DT>(v.x * inv * g.x)) |
+                                    (static_cast<uint32_t>(float_to_bits<DT>(v.y * inv * g.y)) << 16);
+                const uint32_t hi = static_cast<uint32_t>(float_to_bits<DT>(v.z * inv * g.z)) |
+                                    (static_cast<uint32_t>(float_to_bits<DT>(v.w * inv * g.w)) << 16);
+                reinterpret_cast<uint2*>(xs + static_cast<size_t>(t) * Kp)[c] = make_uint2(lo, hi);
+                if (scribe && a.xnorm_out != nullptr)
+                    reinterpret_cast<uint2*>(a.xnorm_out + static_cast<size_t>(t) * K)[c] = make_uint2(lo, hi);
+            };
+#pragma unroll
+            for (int i = 0; i < NH; ++i) {
+                const int c = tid + i * kGemvThreads;
+                if (c < nq) emit(c, hv[i]);
             }
+            for (int c = tid + NH * kGemvThreads; c < nq; c += kGemvThreads) emit(c, ht[c]);
         }
         __syncthreads();
-        xin = xs;
     }
+    // 16-bit input of token t, channel j, once the stage above / below has run
+    auto x_at = [&](int t, int j) -> uint16_t {
+        if (IN == IN_NORM) return xs[static_cast<size_t>(t) * Kp + j];
+        return T == 1 ? xs[j] : a.x[static_cast<size_t>(t) * K + j];
+    };
+    AFX_MARK(2);
 
     // ---- selection ----------------------------------------------------------------------
-    int cnt;
-    int warp_base = 0;  // position of this warp's first active channel in the list
-    int w0 = 0, w1 = 0;
-    const bool own = (a.idx_in == nullptr);
+    int cnt = 0;
+    int pos0 = 0;                  // list position of this thread's first active channel
+    unsigned long long fl = 0ull;  // this thread's active flags (own selection)
     if (own) {
-        block_select_flags<DT>(xin, K, T, a.mode, a.k, a.tau, flags, sel);
-        warp_word_range(nwords, w0, w1);
-        int c = 0;
-        for (int w = w0 + lane; w < w1; w += 32) c += __popc(flags[w]);
-        c = warp_sum(c);
-        warp_base = block_exclusive_over_warps(c, sel->scan);
-        cnt = sel->scan[32];
+        for (int t = 0; t < T; ++t) {
+            const uint16_t* xt = xs + (IN == IN_NORM ? static_cast<size_t>(t) * Kp : 0);
+            if (IN == IN_X) {
+                if (t > 0) __syncthreads();  // the previous token's keys are still being read
+                block_stage_token(a.x + static_cast<size_t>(t) * K, K, xs);
+            }
+            fl |= block_token_flags<DT, kGemvThreads>(xt, K, a.mode, a.k, a.tau, hist, t == 0, sel, T == 1,
+                                                      pos0, cnt);
+        }
+        if (T > 1) pos0 = block_prefix(__popcll(fl), sel->wtot[2], cnt);
+        if (scribe) store_flag_bytes(fl, K, flags);
     } else {
+        if (IN == IN_X && T == 1) block_stage_token(a.x, K, xs);
         cnt = *a.count_in;
         cnt = max(0, min(cnt, K));
     }
-    const int c_lo = static_cast<int>(static_cast<int64_t>(s) * cnt / S);
-    const int c_hi = static_cast<int>(static_cast<int64_t>(s + 1) * cnt / S);
+    AFX_MARK(3);
+    const int c_lo = s * cnt / S;  // S <= 8, cnt <= 2^20: no overflow
+    const int c_hi = (s + 1) * cnt / S;
     const int out0 = tile * PW + (lane % LPC) * 8;
     const bool lane_ok = out0 < a.N;
-    const uint32_t lt_mask = (1u << lane) - 1u;
 
     float acc[TMAX][8];
 #pragma unroll
@@ -123,65 +176,52 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
 
     for (int c0 = c_lo; c0 < c_hi; c0 += CAP) {
         const int staged = min(CAP, c_hi - c0);
-        __syncthreads();
+        __syncthreads();  // the work area is free: the histogram / the previous stage has been read
         // ---- stage (column, x values) of list positions [c0, c0 + staged) ----
         if (own) {
-            int base = warp_base;
-            for (int w = w0; w < w1; ++w) {
-                const uint32_t bits = flags[w];
-                const int n = __popc(bits);
-                if (base + n > c0 && base < c0 + staged && ((bits >> lane) & 1u)) {
-                    const int pos = base + __popc(bits & lt_mask) - c0;
-                    if (pos >= 0 && pos < staged) {
-                        const int j = (w << 5) + lane;
-                        sm->col[pos] = j;
+            for_each_owned_active(fl, K, pos0, [&](int j, int pos) {
+                const int p = pos - c0;
+                if (p >= 0 && p < staged) {
+                    sm->col[p] = j;
 #pragma unroll
-                        for (int t = 0; t < TMAX; ++t)
-                            if (t < T) sm->xv[t][pos] = bits_to_float<DT>(xin[static_cast<size_t>(t) * K + j]);
-                    }
+                    for (int t = 0; t < TMAX; ++t)
+                        if (t < T) sm->xv[t][p] = bits_to_float<DT>(x_at(t, j));
                 }
-                base += n;
-            }
+            });
         } else {
             for (int i = tid; i < staged; i += kGemvThreads) {
                 const int j = a.idx_in[c0 + i];
                 sm->col[i] = j;
 #pragma unroll
                 for (int t = 0; t < TMAX; ++t)
-                    if (t < T) sm->xv[t][i] = bits_to_float<DT>(xin[static_cast<size_t>(t) * K + j]);
+                    if (t < T) sm->xv[t][i] = bits_to_float<DT>(x_at(t, j));
             }
         }
         __syncthreads();
+        AFX_MARK(4);
         if (lane_ok) gemv_stream<DT, TMAX, PW, CAP>(a.Wt + out0, a.ldw, T, sm, staged, acc);
     }
+    AFX_MARK(5);
 
     // ---- side outputs (one block of the grid) ---------------------------------------------
     if (scribe) {
         if (own) {
-            if (a.idx_out != nullptr) {
-                int base = warp_base;
-                for (int w = w0; w < w1; ++w) {
-                    const uint32_t bits = flags[w];
-                    if ((bits >> lane) & 1u) a.idx_out[base + __popc(bits & lt_mask)] = (w << 5) + lane;
-                    base += __popc(bits);
-                }
-            }
+            if (a.idx_out != nullptr) for_each_owned_active(fl, K, pos0, [&](int j, int pos) { a.idx_out[pos] = j; });
+            __syncthreads();  // flag bytes of every thread are in place
             if (a.bitmap_out != nullptr)
                 for (int w = tid; w < nwords; w += kGemvThreads) a.bitmap_out[w] = flags[w];
             if (a.bitmap_pred != nullptr) {
-                // A \ P in ascending order, |A & P|
-                int c = 0;
-                for (int w = w0 + lane; w < w1; w += 32) c += __popc(flags[w] & ~a.bitmap_pred[w]);
-                c = warp_sum(c);
-                int base = block_exclusive_over_warps(c, sel->scan);
-                const int n_miss = sel->scan[32];
-                if (a.miss_out != nullptr) {
-                    for (int w = w0; w < w1; ++w) {
-                        const uint32_t bits = flags[w] & ~a.bitmap_pred[w];
-                        if ((bits >> lane) & 1u) a.miss_out[base + __popc(bits & lt_mask)] = (w << 5) + lane;
-                        base += __popc(bits);
-                    }
-                }
+                // A \ P in ascending order, |A & P|: the predicted set, byte by byte like fl
+                int q_lo, q_hi;
+                thread_chunk_range(K, q_lo, q_hi);
+                const uint8_t* pred = reinterpret_cast<const uint8_t*>(a.bitmap_pred);
+                unsigned long long pm = 0ull;
+                for (int c = q_lo; c < q_hi; ++c) pm |= static_cast<unsigned long long>(pred[c]) << (8 * (c - q_lo));
+                const unsigned long long ms = fl & ~pm;
+                int n_miss;
+                const int m0 = block_prefix(__popcll(ms), sel->wtot[3], n_miss);
+                if (a.miss_out != nullptr)
+                    for_each_owned_active(ms, K, m0, [&](int j, int pos) { a.miss_out[pos] = j; });
                 if (tid == 0) {
                     if (a.miss_count != nullptr) *a.miss_count = n_miss;
                     if (a.hit_count != nullptr) *a.hit_count = cnt - n_miss;
@@ -192,8 +232,10 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
         }
         if (tid == 0 && a.count_out != nullptr) *a.count_out = cnt;
     }
+    AFX_MARK(6);
 
     gemv_finish_tile<DT, TMAX, PW, CAP, EP>(acc, T, tile, sm, a.ep);
+    AFX_MARK(7);
 }
 
 }  // namespace afx

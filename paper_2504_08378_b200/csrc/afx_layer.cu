@@ -20,15 +20,22 @@ __global__ void __launch_bounds__(kGemvThreads, FusedShape<TMAX>::kBlocksPerSM)
 fused_op_kernel(FusedArgs a) {
     constexpr int CAP = FusedShape<TMAX>::kStageCap;
     extern __shared__ __align__(16) unsigned char dyn[];
-    __shared__ GemvSmem<TMAX, CAP> sm;
     __shared__ SelectScratch sel;
-    fused_op_block<DT, TMAX, PW, CAP, IN, EP>(a, dyn, &sm, &sel);
+    fused_op_block<DT, TMAX, PW, CAP, IN, EP>(a, dyn, &sel);
+}
+
+template <int DT, int REP>
+__global__ void __launch_bounds__(kAttnThreads, REP <= 2 ? 2 : 1) attention_kernel(AttnArgs a) {
+    __shared__ AttnSmem sm;
+    attention_block<DT, REP>(a, &sm);
 }
 
 template <int DT>
-__global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(AttnArgs a) {
-    __shared__ AttnSmem sm;
-    attention_block<DT>(a, &sm);
+static cudaError_t launch_attention_rep(const cudaLaunchConfig_t& cfg, int rep, const AttnArgs& a) {
+    if (rep <= 1) return cudaLaunchKernelEx(&cfg, attention_kernel<DT, 1>, a);
+    if (rep <= 2) return cudaLaunchKernelEx(&cfg, attention_kernel<DT, 2>, a);
+    if (rep <= 4) return cudaLaunchKernelEx(&cfg, attention_kernel<DT, 4>, a);
+    return cudaLaunchKernelEx(&cfg, attention_kernel<DT, 8>, a);
 }
 
 template <int DT, int TMAX, int IN, int EP>
@@ -75,8 +82,9 @@ static afx_status launch_attention(int dtype, const AttnArgs& a, cudaStream_t st
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    const cudaError_t e = dtype == AFX_F16 ? cudaLaunchKernelEx(&cfg, attention_kernel<AFX_F16>, a)
-                                           : cudaLaunchKernelEx(&cfg, attention_kernel<AFX_BF16>, a);
+    const int rep = a.q_heads / a.kv_heads;
+    const cudaError_t e = dtype == AFX_F16 ? launch_attention_rep<AFX_F16>(cfg, rep, a)
+                                           : launch_attention_rep<AFX_BF16>(cfg, rep, a);
     return e == cudaSuccess ? AFX_OK : AFX_ERR_CUDA;
 }
 
@@ -155,7 +163,7 @@ extern "C" afx_status afx_model_create(const afx_model_desc* desc, const afx_lay
             L.g_attn == nullptr || L.g_mlp == nullptr || L.k_cache == nullptr || L.v_cache == nullptr)
             return AFX_ERR_INVALID_ARG;
         if (!aligned16(L.w_qkv) || !aligned16(L.w_o) || !aligned16(L.w_gu) || !aligned16(L.w_down) ||
-            !aligned16(L.k_cache) || !aligned16(L.v_cache))
+            !aligned16(L.k_cache) || !aligned16(L.v_cache) || !aligned16(L.g_attn) || !aligned16(L.g_mlp))
             return AFX_ERR_ALIGNMENT;
         for (int op = 0; op < 4; ++op) {
             if (d.select_mode == AFX_MODE_TOPK && (L.k[op] < 0 || L.k[op] > K_op[op])) return AFX_ERR_INVALID_ARG;
@@ -215,7 +223,8 @@ extern "C" afx_status afx_state_create(const afx_model* model, int T, void* blob
     }
     // the widest input stage must fit one block's shared memory
     const size_t dyn_max = afx::fused_dyn_smem(afx::IN_NORM, model->d.hidden, T);
-    if (dyn_max > 160 * 1024) {
+    if (dyn_max > 200 * 1024 || model->d.mlp > afx::kSelectFastMaxK ||
+        model->d.n_heads * model->d.head_dim > afx::kSelectFastMaxK) {
         delete s;
         return AFX_ERR_UNSUPPORTED;
     }
@@ -431,7 +440,8 @@ extern "C" afx_status afx_select_gemv(const void* Wt, int dtype, int K, int N, i
                                       int32_t* count_out, void* stream) {
     using namespace afx;
     if (Wt == nullptr || x == nullptr || y == nullptr) return AFX_ERR_INVALID_ARG;
-    if (K <= 0 || K > (1 << 20) || N <= 0 || T < 1 || T > AFX_MAX_T || ldw < N) return AFX_ERR_INVALID_ARG;
+    if (K <= 0 || N <= 0 || T < 1 || T > AFX_MAX_T || ldw < N) return AFX_ERR_INVALID_ARG;
+    if (K > kSelectFastMaxK) return AFX_ERR_CAPACITY;
     if (dtype != AFX_F16 && dtype != AFX_BF16) return AFX_ERR_UNSUPPORTED;
     if (mode != AFX_MODE_TOPK && mode != AFX_MODE_THRESHOLD) return AFX_ERR_UNSUPPORTED;
     if (mode == AFX_MODE_TOPK && (k < 0 || k > K)) return AFX_ERR_INVALID_ARG;

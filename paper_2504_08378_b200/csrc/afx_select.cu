@@ -1,23 +1,69 @@
 // afx_select_active / afx_diff_active: stand-alone selection and cross-layer set difference.
+#include "afx_launch.cuh"
 #include "afx_select.cuh"
 
 namespace afx {
 
 constexpr int kSelectThreads = 1024;
 
+// Dynamic shared memory.  Fast path: [flag words, padded to 16 bytes] [one token's keys] [key
+// histogram].  Large-K path: flag words only.
+static size_t select_dyn_smem(int K) {
+    size_t b = (static_cast<size_t>((K + 31) >> 5) * 4 + 15) / 16 * 16;
+    if (K <= kSelectFastMaxK) b += (static_cast<size_t>(K) + 7) / 8 * 8 * 2 + kKeyHistBytes;
+    return b;
+}
+
 template <int DT>
 __global__ void __launch_bounds__(kSelectThreads, 1)
 select_kernel(const uint16_t* __restrict__ x, int K, int T, int mode, int k, float tau,
               int32_t* __restrict__ idx, int32_t* __restrict__ count, uint32_t* __restrict__ bitmap) {
-    extern __shared__ uint32_t s_flags[];
+    extern __shared__ __align__(16) unsigned char s_dyn[];
     __shared__ SelectScratch scratch;
-    block_select_flags<DT>(x, K, T, mode, k, tau, s_flags, &scratch);
-    const int total = block_compact_flags(s_flags, K, idx, &scratch);
-    if (threadIdx.x == 0) *count = total;
-    if (bitmap != nullptr) {
-        const int nwords = (K + 31) >> 5;
-        for (int w = threadIdx.x; w < nwords; w += blockDim.x) bitmap[w] = s_flags[w];
+    const int nwords = (K + 31) >> 5;
+    const size_t flag_bytes = (static_cast<size_t>(nwords) * 4 + 15) / 16 * 16;
+    uint32_t* s_flags = reinterpret_cast<uint32_t*>(s_dyn);
+    const int lane = lane_id();
+    if (K <= kSelectFastMaxK) {
+        uint16_t* xs = reinterpret_cast<uint16_t*>(s_dyn + flag_bytes);
+        uint32_t* hist = reinterpret_cast<uint32_t*>(s_dyn + flag_bytes + (static_cast<size_t>(K) + 7) / 8 * 8 * 2);
+        const bool topk = mode == AFX_MODE_TOPK && k > 0 && k < K;
+        if (topk) block_clear_key_hist(hist);
+        unsigned long long fl = 0ull;
+        int pos0 = 0, total = 0;
+        for (int t = 0; t < T; ++t) {
+            if (t > 0) __syncthreads();  // the previous token's keys are still being read
+            block_stage_token(x + static_cast<size_t>(t) * K, K, xs);
+            fl |= block_token_flags<DT, kSelectThreads>(xs, K, mode, k, tau, hist, t == 0, &scratch, T == 1,
+                                                        pos0, total);
+        }
+        if (T > 1) pos0 = block_prefix(__popcll(fl), scratch.wtot[2], total);
+        for_each_owned_active(fl, K, pos0, [&](int j, int pos) { idx[pos] = j; });
+        if (threadIdx.x == 0) *count = total;
+        if (bitmap != nullptr) {
+            store_flag_bytes(fl, K, s_flags);
+            __syncthreads();
+            for (int w = threadIdx.x; w < nwords; w += blockDim.x) bitmap[w] = s_flags[w];
+        }
+        return;
     }
+    int w0, w1;
+    warp_word_range(nwords, w0, w1);
+    int mine = 0;
+    block_select_flags_large<DT>(x, K, T, mode, k, tau, s_flags, &scratch);
+    for (int w = w0 + lane; w < w1; w += 32) mine += __popc(s_flags[w]);
+    mine = warp_sum(mine);
+    int total;
+    int base = warp_prefix(mine, scratch.wtot[1], total);
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    for (int w = w0; w < w1; ++w) {
+        const uint32_t bits = s_flags[w];
+        if ((bits >> lane) & 1u) idx[base + __popc(bits & lt_mask)] = (w << 5) + lane;
+        base += __popc(bits);
+    }
+    if (threadIdx.x == 0) *count = total;
+    if (bitmap != nullptr)
+        for (int w = w0 + lane; w < w1; w += 32) bitmap[w] = s_flags[w];
 }
 
 // miss = A \ P (ascending), hit = |A & P|.  One block; each warp owns a contiguous run of
@@ -45,8 +91,8 @@ diff_kernel(const int32_t* __restrict__ idxA, const int32_t* __restrict__ cntA,
         }
         cm += __popc(__ballot_sync(0xFFFFFFFFu, m));
     }
-    int base = block_exclusive_over_warps(cm, scan);
-    const int total = scan[32];
+    int total;
+    int base = warp_prefix(cm, scan, total);
     for (int c = c0; c < c1; ++c) {
         const int p = (c << 5) + lane;
         bool m = false;
@@ -80,12 +126,11 @@ extern "C" afx_status afx_select_active(const void* x, int dtype, int K, int T, 
     if ((reinterpret_cast<uintptr_t>(x) & 1u) || (reinterpret_cast<uintptr_t>(idx) & 3u) ||
         (reinterpret_cast<uintptr_t>(count) & 3u) || (reinterpret_cast<uintptr_t>(bitmap) & 3u))
         return AFX_ERR_ALIGNMENT;
-    const size_t smem = static_cast<size_t>((K + 31) >> 5) * sizeof(uint32_t);
+    const size_t smem = select_dyn_smem(K);
     auto kern = dtype == AFX_F16 ? select_kernel<AFX_F16> : select_kernel<AFX_BF16>;
-    if (smem > 40 * 1024) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(smem)) != cudaSuccess)
-            return AFX_ERR_CUDA;
+    if (!ensure_dyn_smem(reinterpret_cast<const void*>(kern), smem)) {
+        cudaGetLastError();
+        return AFX_ERR_CUDA;
     }
     kern<<<1, kSelectThreads, smem, static_cast<cudaStream_t>(stream)>>>(
         static_cast<const uint16_t*>(x), K, T, mode, k, tau, idx, count, bitmap);

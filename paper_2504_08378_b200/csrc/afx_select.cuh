@@ -1,8 +1,17 @@
-// Block-level active-channel selection: |x| top-k (two-pass radix select on the 15-bit
-// magnitude key, ties to the lower channel id) or threshold, OR-ed over T tokens into a
-// shared-memory bitmap, then an ordered compaction into an ascending index list.
+// Block-level active-channel selection: |x| top-k (ties to the lower channel id) or threshold,
+// OR-ed over T tokens, then an ordered compaction into an ascending index list.
 //
-// The routines are written for one thread block of whole warps (<= 32 warps) so that the
+// Fast path (K <= 32768, one token's 16-bit patterns in shared memory).  Every thread owns a
+// contiguous run of 8-channel chunks, so "ascending channel id" is "ascending thread id" and
+// one block-wide prefix scan orders both the tie-break and the compaction.  Top-k finds the
+// k-th largest 15-bit magnitude key in ONE counting pass: a full histogram of the 32768
+// possible keys (16-bit counters, 64 KB of shared memory) filled with shared-memory atomics
+// -- real-valued activations spread over hundreds of distinct keys, so the atomics rarely
+// collide, where a histogram of the high key bits alone would serialise on a few exponent
+// bins -- followed by a top-down search: per-warp totals, the warp that holds the k-th key,
+// the row, the lane, the counter.
+//
+// The routines are written for one thread block of 256, 512 or 1024 threads so that the
 // stand-alone selection kernel and kernels that need the selection as a prologue can share
 // them.  Every routine contains block-wide barriers: all threads of the block call it with
 // the same arguments.
@@ -12,14 +21,19 @@
 
 namespace afx {
 
+constexpr int kSelectFastMaxK = 32768;  // keys of one token held in shared memory
+constexpr int kKeyHistWords = 16384;    // 32768 16-bit counters
+constexpr size_t kKeyHistBytes = static_cast<size_t>(kKeyHistWords) * 4;
+
 struct SelectScratch {
-    int hist[256];
+    int wtot[4][32];  // per-warp totals for the ordered scans
+    int res[4];       // broadcast of the k-th key search
+    int hist[256];    // large-K path; the fused operators borrow it for the norm's reduction
     int scan[33];
-    int res[4];
 };
 
-// Words [w0, w1) of the bitmap owned by the calling warp (contiguous, so that a walk over
-// warps in order visits channels in ascending order).
+// Words [w0, w1) of a ceil(K/32)-word bitmap owned by the calling warp (contiguous, so that
+// a walk over warps in order visits channels in ascending order).
 __device__ __forceinline__ void warp_word_range(int nwords, int& w0, int& w1) {
     const int nw = blockDim.x >> 5;
     const int per = (nwords + nw - 1) / nw;
@@ -27,6 +41,282 @@ __device__ __forceinline__ void warp_word_range(int nwords, int& w0, int& w1) {
     w1 = min(nwords, w0 + per);
     if (w0 > nwords) w0 = nwords;
 }
+
+// Exclusive prefix over the warps of the block of one int per warp (`mine`, same in all
+// lanes); `total` receives the block's sum.  One barrier.  `buf` (32 ints of shared memory)
+// must not be written again before every warp has passed a later barrier.
+__device__ __forceinline__ int warp_prefix(int mine, int* buf, int& total) {
+    const int nw = blockDim.x >> 5;
+    const int lane = lane_id();
+    if (lane == 0) buf[warp_id()] = mine;
+    __syncthreads();
+    const int v = lane < nw ? buf[lane] : 0;
+    int incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int n = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += n;
+    }
+    total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+    return __shfl_sync(0xFFFFFFFFu, incl - v, warp_id());
+}
+
+// Exclusive prefix over the THREADS of the block (thread order) of `v`; `total` = block sum.
+__device__ __forceinline__ int block_prefix(int v, int* buf, int& total) {
+    const int lane = lane_id();
+    int incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int n = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += n;
+    }
+    const int wsum = __shfl_sync(0xFFFFFFFFu, incl, 31);
+    return warp_prefix(wsum, buf, total) + incl - v;
+}
+
+// The chunks (8 channels each) owned by the calling thread: [c_lo, c_hi), at most 8.
+__device__ __forceinline__ void thread_chunk_range(int K, int& c_lo, int& c_hi) {
+    const int nchunks = (K + 7) >> 3;
+    const int m = (nchunks + blockDim.x - 1) / blockDim.x;
+    c_lo = min(static_cast<int>(threadIdx.x) * m, nchunks);
+    c_hi = min(c_lo + m, nchunks);
+}
+
+__device__ __forceinline__ void chunk_keys(const uint16_t* xs, int c, uint32_t (&key)[8]) {
+    const uint4 raw = *reinterpret_cast<const uint4*>(xs + (c << 3));
+    const uint32_t r[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        key[2 * i] = r[i] & 0x7FFFu;
+        key[2 * i + 1] = (r[i] >> 16) & 0x7FFFu;
+    }
+}
+
+// Sets the key histogram to zero (no barrier).
+__device__ __forceinline__ void block_clear_key_hist(uint32_t* hist) {
+    for (int i = threadIdx.x; i < kKeyHistWords / 4; i += blockDim.x)
+        reinterpret_cast<uint4*>(hist)[i] = make_uint4(0u, 0u, 0u, 0u);
+}
+
+// The k-th largest magnitude key (1 <= k <= K) of xs[0..K) (shared memory, 16-byte aligned,
+// readable up to the next multiple of 8 elements).  `hist` is kKeyHistWords words of shared
+// memory, all zero and visible on entry (block_clear_key_hist + barrier); it is left dirty.
+// Returns the key in `thr`, how many channels with exactly that key belong to the top k in
+// `need_eq`, and how many channels have that key in `tot_eq`.  Same values in every thread.
+template <int NT>
+__device__ __forceinline__ void block_kth_key(const uint16_t* xs, int K, int k, uint32_t* hist,
+                                              SelectScratch* s, uint32_t& thr, int& need_eq, int& tot_eq) {
+    constexpr int NW = NT / 32;
+    constexpr int W = kKeyHistWords / NW;  // histogram words per warp
+    constexpr int NR = W / 128;            // rows of 32 lanes x 4 words
+    static_assert(NR >= 1 && NR * 128 * NW == kKeyHistWords, "block size must be 256, 512 or 1024");
+    const int lane = lane_id();
+    const int warp = warp_id();
+    int c_lo, c_hi;
+    thread_chunk_range(K, c_lo, c_hi);
+    for (int c = c_lo; c < c_hi; ++c) {
+        uint32_t key[8];
+        chunk_keys(xs, c, key);
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+            if ((c << 3) + e < K) atomicAdd(&hist[key[e] >> 1], 1u << ((key[e] & 1u) << 4));
+    }
+    __syncthreads();
+    // counters of this warp's slice, highest keys last: row i, lane l holds words
+    // warp*W + (i*32 + l)*4 .. +4
+    const uint32_t* mine = hist + warp * W + lane * 4;
+    int rowsum[NR];
+    int lane_total = 0;
+#pragma unroll
+    for (int i = 0; i < NR; ++i) {
+        const uint4 v = *reinterpret_cast<const uint4*>(mine + i * 128);
+        const uint32_t p = v.x + v.y + v.z + v.w;  // two 16-bit lanes, neither overflows (K <= 32768)
+        rowsum[i] = static_cast<int>((p & 0xFFFFu) + (p >> 16));
+        lane_total += rowsum[i];
+    }
+    const int warp_total = __reduce_add_sync(0xFFFFFFFFu, lane_total);
+    int total;
+    const int below = warp_prefix(warp_total, s->wtot[0], total);
+    const int above = total - below - warp_total;  // keys in the slices of higher warps
+    if (above < k && k <= above + warp_total) {    // exactly one warp holds the k-th largest key
+        int rem = k - above;                       // rank from the top inside this warp's slice
+        int row = 0, row_lane_sum = 0;
+        bool found = false;
+#pragma unroll
+        for (int i = NR - 1; i >= 0; --i) {
+            const int rt = __reduce_add_sync(0xFFFFFFFFu, rowsum[i]);
+            if (!found) {
+                if (rem <= rt) {
+                    found = true;
+                    row = i;
+                    row_lane_sum = rowsum[i];
+                } else {
+                    rem -= rt;
+                }
+            }
+        }
+        // inclusive suffix sums over the lanes of that row (higher lanes hold higher keys)
+        int suf = row_lane_sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int n = __shfl_down_sync(0xFFFFFFFFu, suf, o);
+            if (lane + o < 32) suf += n;
+        }
+        const uint32_t ok = __ballot_sync(0xFFFFFFFFu, suf >= rem);
+        const int l_star = 31 - __clz(static_cast<int>(ok));
+        if (lane == l_star) {
+            rem -= suf - row_lane_sum;  // keys in higher lanes of the row
+            const uint4 v = *reinterpret_cast<const uint4*>(mine + row * 128);
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+            const int word0 = warp * W + (row * 32 + lane) * 4;
+            bool done = false;
+#pragma unroll
+            for (int q = 3; q >= 0; --q) {
+#pragma unroll
+                for (int h = 1; h >= 0; --h) {
+                    const int c = static_cast<int>((w[q] >> (16 * h)) & 0xFFFFu);
+                    if (!done) {
+                        if (rem <= c) {
+                            done = true;
+                            s->res[0] = 2 * (word0 + q) + h;
+                            s->res[1] = rem;
+                            s->res[2] = c;
+                        } else {
+                            rem -= c;
+                        }
+                    }
+                }
+            }
+        }
+    }
+    __syncthreads();
+    thr = static_cast<uint32_t>(s->res[0]);
+    need_eq = s->res[1];
+    tot_eq = s->res[2];
+}
+
+// Active flags of ONE token for the calling thread's chunks: byte v of the result covers the
+// 8 channels of chunk c_lo + v (bit e = channel 8 * (c_lo + v) + e).  xs as for
+// block_kth_key.  `hist` is the key histogram (top-k only); `hist_clean` says that it is
+// already zero and visible.  With `single` set (the token is the only one) the call also
+// returns the list position of the thread's first active channel in `pos0` and the length
+// of the list in `cnt`, from the same scan that orders the tie-break.
+template <int DT, int NT>
+__device__ __forceinline__ unsigned long long block_token_flags(const uint16_t* xs, int K, int mode, int k,
+                                                                float tau, uint32_t* hist, bool hist_clean,
+                                                                SelectScratch* s, bool single, int& pos0,
+                                                                int& cnt) {
+    int c_lo, c_hi;
+    thread_chunk_range(K, c_lo, c_hi);
+    unsigned long long fl = 0ull;
+    if (mode == AFX_MODE_THRESHOLD || k >= K || k <= 0) {
+        const bool all = mode == AFX_MODE_THRESHOLD ? tau < 0.0f : k > 0;
+        const bool none = mode != AFX_MODE_THRESHOLD && k <= 0;
+        for (int c = c_lo; c < c_hi; ++c) {
+            const uint4 raw = *reinterpret_cast<const uint4*>(xs + (c << 3));
+            const uint32_t r[4] = {raw.x, raw.y, raw.z, raw.w};
+            uint32_t byte = 0;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const uint16_t bits = static_cast<uint16_t>(r[e >> 1] >> (16 * (e & 1)));
+                const bool in = (c << 3) + e < K;
+                const bool pred = in && !none && (all || fabsf(bits_to_float<DT>(bits)) > tau);
+                byte |= static_cast<uint32_t>(pred) << e;
+            }
+            fl |= static_cast<unsigned long long>(byte) << (8 * (c - c_lo));
+        }
+        if (single) pos0 = block_prefix(__popcll(fl), s->wtot[1], cnt);
+        return fl;
+    }
+    if (!hist_clean) {
+        block_clear_key_hist(hist);
+        __syncthreads();
+    }
+    uint32_t thr;
+    int need_eq, tot_eq;
+    block_kth_key<NT>(xs, K, k, hist, s, thr, need_eq, tot_eq);
+    // channels above the k-th key are in; of those equal to it, the need_eq lowest ids
+    int g = 0, e_cnt = 0;
+    for (int c = c_lo; c < c_hi; ++c) {
+        uint32_t key[8];
+        chunk_keys(xs, c, key);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const bool in = (c << 3) + e < K;
+            g += in && key[e] > thr;
+            e_cnt += in && key[e] == thr;
+        }
+    }
+    int pre_e = 0;
+    if (single) {
+        int tot;
+        const int pre = block_prefix((g << 16) | e_cnt, s->wtot[1], tot);  // g < 2^15, e <= 2^15: no carry
+        pre_e = pre & 0xFFFF;
+        pos0 = (pre >> 16) + min(pre_e, need_eq);
+        cnt = k;
+    } else if (need_eq != tot_eq) {
+        int tot;
+        pre_e = block_prefix(e_cnt, s->wtot[1], tot);
+    }
+    int seen_e = pre_e;
+    for (int c = c_lo; c < c_hi; ++c) {
+        uint32_t key[8];
+        chunk_keys(xs, c, key);
+        uint32_t byte = 0;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const bool in = (c << 3) + e < K;
+            const bool eq = in && key[e] == thr;
+            const bool pred = in && (key[e] > thr || (eq && (need_eq == tot_eq || seen_e < need_eq)));
+            seen_e += eq;
+            byte |= static_cast<uint32_t>(pred) << e;
+        }
+        fl |= static_cast<unsigned long long>(byte) << (8 * (c - c_lo));
+    }
+    return fl;
+}
+
+// Writes the calling thread's flag bytes into a ceil(K/32)-word bitmap in shared memory
+// (bit j % 32 of word j / 32) and clears the bytes past the last chunk.  No barrier.
+__device__ __forceinline__ void store_flag_bytes(unsigned long long fl, int K, uint32_t* flags) {
+    int c_lo, c_hi;
+    thread_chunk_range(K, c_lo, c_hi);
+    uint8_t* bytes = reinterpret_cast<uint8_t*>(flags);
+    for (int c = c_lo; c < c_hi; ++c) bytes[c] = static_cast<uint8_t>(fl >> (8 * (c - c_lo)));
+    const int nchunks = (K + 7) >> 3, nbytes = ((K + 31) >> 5) << 2;
+    for (int c = nchunks + threadIdx.x; c < nbytes; c += blockDim.x) bytes[c] = 0;
+}
+
+// Calls f(j, pos) for every active channel j of the calling thread, ascending, pos = its
+// position in the list.
+template <class F>
+__device__ __forceinline__ void for_each_owned_active(unsigned long long fl, int K, int pos0, F f) {
+    int c_lo, c_hi;
+    thread_chunk_range(K, c_lo, c_hi);
+    int pos = pos0;
+    while (fl != 0ull) {
+        const int b = __ffsll(static_cast<long long>(fl)) - 1;
+        fl &= fl - 1ull;
+        f((c_lo << 3) + b, pos++);
+    }
+}
+
+// Copies one token's K 16-bit patterns from global memory into shared memory and zero-fills
+// up to the next multiple of 8 elements.  Ends with a block barrier.
+__device__ __forceinline__ void block_stage_token(const uint16_t* __restrict__ x, int K, uint16_t* xs) {
+    const int Kp = (K + 7) & ~7;
+    if ((reinterpret_cast<uintptr_t>(x) & 15u) == 0) {
+        const int nfull = K >> 3;
+        for (int c = threadIdx.x; c < nfull; c += blockDim.x)
+            reinterpret_cast<uint4*>(xs)[c] = reinterpret_cast<const uint4*>(x)[c];
+        for (int j = (nfull << 3) + threadIdx.x; j < Kp; j += blockDim.x) xs[j] = j < K ? x[j] : uint16_t(0);
+    } else {
+        for (int j = threadIdx.x; j < Kp; j += blockDim.x) xs[j] = j < K ? x[j] : uint16_t(0);
+    }
+    __syncthreads();
+}
+
+// ---- large-K path (K > kSelectFastMaxK): keys read from global memory ----
 
 // Warp 0 only.  hist has nbins (multiple of 32, <= 256) counters; walking bins from the
 // highest down, finds the bin that holds the k-th element (k is 1-based and must not
@@ -59,10 +349,10 @@ __device__ __forceinline__ void find_kth_bin(const int* hist, int nbins, int k, 
     }
 }
 
-// Fills flags[0..ceil(K/32)) (shared memory) with the union over tokens of the per-token
-// active sets.  x is [T][K] in global memory.
+// Large-K path: fills flags[0..ceil(K/32)) (shared memory) with the union over tokens of the
+// per-token active sets.  x is [T][K] in global memory; two histogram passes per token.
 template <int DT>
-__device__ void block_select_flags(const uint16_t* __restrict__ x, int K, int T, int mode, int k,
+__device__ void block_select_flags_large(const uint16_t* __restrict__ x, int K, int T, int mode, int k,
                                    float tau, uint32_t* flags, SelectScratch* s) {
     const int nwords = (K + 31) >> 5;
     const int lane = lane_id();
@@ -144,28 +434,6 @@ __device__ void block_select_flags(const uint16_t* __restrict__ x, int K, int T,
         }
     }
     __syncthreads();
-}
-
-// Ordered compaction of a bitmap in shared memory: idx[0..total) = set bits ascending.
-// idx may point to global or shared memory.  Returns the total (same in every thread).
-__device__ __forceinline__ int block_compact_flags(const uint32_t* flags, int K, int32_t* idx,
-                                                   SelectScratch* s) {
-    const int nwords = (K + 31) >> 5;
-    const int lane = lane_id();
-    const uint32_t lt_mask = (1u << lane) - 1u;
-    int w0, w1;
-    warp_word_range(nwords, w0, w1);
-    int c = 0;
-    for (int w = w0 + lane; w < w1; w += 32) c += __popc(flags[w]);
-    c = warp_sum(c);
-    int base = block_exclusive_over_warps(c, s->scan);
-    const int total = s->scan[32];
-    for (int w = w0; w < w1; ++w) {
-        const uint32_t bits = flags[w];
-        if ((bits >> lane) & 1u) idx[base + __popc(bits & lt_mask)] = (w << 5) + lane;
-        base += __popc(bits);
-    }
-    return total;
 }
 
 }  // namespace afx
