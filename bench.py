@@ -30,10 +30,10 @@ sys.path.insert(0, ROOT)
 
 CFG = dict(name="llama7b_decode_32L_bf16_top50_xl3", dtype="bf16", n_layers=32, hidden=4096, n_heads=32,
            n_kv_heads=32, mlp=11008, past=2048, sparsity_percent=50, xl_depth=3, seed=3)
-ORACLE_SAMPLE_LAYERS = 2
+ORACLE_SAMPLE_LAYERS = 16
 # dram__bytes_read.sum + dram__bytes_write.sum of one fused gate/up launch of this workload,
-# from the ncu capture summarised under profiles/ (None until captured).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+# from the ncu capture summarised in profiles/fused_op_kernel_7b_ncu_full.md (None when stale).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 94_080_256
 
 
 def measured_peaks():
@@ -157,7 +157,10 @@ def run_afx(args):
 
     world, rank, local = dist_setup(args.gpus)
     torch.cuda.set_device(local)
-    cfg = CFG
+    cfg = dict(CFG)
+    if args.layers:  # reduced stack for profiler captures; the JSON line says so
+        cfg["n_layers"] = args.layers
+        cfg["name"] = CFG["name"] + f"_first{args.layers}layers"
     m, layers, k = build_model(cfg)
     pos = cfg["past"]
     h0_host = torch.from_numpy(synth.hidden_state(cfg["seed"], 5, 1, cfg["hidden"], scale=1.0,
@@ -292,7 +295,7 @@ def cpu_baseline(cfg, layers, k, h0, pos):
     import oracle
     import oracle.layer as ol
     from paper_2504_08378_b200 import synth
-    n = ORACLE_SAMPLE_LAYERS
+    n = min(ORACLE_SAMPLE_LAYERS, cfg["n_layers"])
     ocfg = ol.Config(cfg["dtype"], cfg["hidden"], cfg["n_heads"], cfg["n_kv_heads"], cfg["mlp"], mode=oracle.TOPK)
     lws, caches = [], []
     for l in range(n):
@@ -370,6 +373,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="afx", choices=["afx", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="run only the first N layers (profiling aid)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
