@@ -53,7 +53,8 @@ __host__ __device__ inline size_t fused_dyn_smem(int in_kind, int K, int T) {
 }
 
 template <int DT, int TMAX, int PW, int CAP, int IN, int EP>
-__device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char* dyn, SelectScratch* sel) {
+__device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char* dyn, SelectScratch* sel,
+                                               GemvRecv<TMAX>* recv) {
     constexpr int LPC = PW / 8;
     static_assert(sizeof(GemvSmem<TMAX, CAP>) <= kKeyHistBytes, "work area too small");
     const int tid = threadIdx.x;
@@ -75,6 +76,7 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
     const bool own = (a.idx_in == nullptr);
     const bool topk = own && a.mode == AFX_MODE_TOPK && a.k > 0 && a.k < K;
     AFX_MARK(0);
+    cluster_arrive();
     if (topk) block_clear_key_hist(hist);  // does not depend on the previous kernel
 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -234,7 +236,7 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
     }
     AFX_MARK(6);
 
-    gemv_finish_tile<DT, TMAX, PW, CAP, EP>(acc, T, tile, sm, a.ep);
+    gemv_finish_tile<DT, TMAX, PW, CAP, EP>(acc, T, tile, sm, recv, a.ep);
     AFX_MARK(7);
 }
 

@@ -14,7 +14,8 @@ __global__ void __launch_bounds__(kGemvThreads, GemvShape<TMAX>::kBlocksPerSM)
 sparse_gemv_kernel(GemvListArgs a) {
     constexpr int CAP = GemvShape<TMAX>::kStageCap;
     __shared__ GemvSmem<TMAX, CAP> sm;
-    gemv_list_block<DT, TMAX, PW, CAP>(a, &sm);
+    __shared__ GemvRecv<TMAX> recv;
+    gemv_list_block<DT, TMAX, PW, CAP>(a, &sm, &recv);
 }
 
 int sm_count() {

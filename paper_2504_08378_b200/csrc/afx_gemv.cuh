@@ -30,8 +30,26 @@ struct GemvSmem {
     int col[CAP];
     float xv[TMAX][CAP];
     __align__(16) float red[kGemvWarps][256];  // per-warp sums of one token
-    __align__(16) float part[TMAX][256];       // this block's sums, read by the cluster
 };
+
+// Where the blocks of a cluster deliver their partial sums: block q owns every S-th output
+// (or gate/up pair) of the tile and receives one value per (source block, token, owned
+// output).  Written by remote blocks while this block may still be in any phase of its own
+// work, so it must not share storage with anything else.
+constexpr int kRecvPerToken = 272;  // >= PW + 2 * kMaxCluster - 2
+template <int TMAX>
+struct GemvRecv {
+    float v[TMAX * kRecvPerToken];
+};
+
+// Split cluster barrier.  Every block arrives once when it starts and waits just before its
+// first store into a peer's shared memory: by then every block of the cluster is running.
+__device__ __forceinline__ void cluster_arrive() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait() {
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 
 // How a finished sum leaves the kernel.
 enum { EP_STORE = 0, EP_ACCUM = 1, EP_SILU = 2 };
@@ -83,17 +101,37 @@ __device__ __forceinline__ void gemv_stream(const uint16_t* __restrict__ wbase, 
 //   EP_STORE  y[t][out]  = sum            EP_ACCUM  y[t][out] += sum
 //   EP_SILU   columns come in groups of 16 = 8 "gate" then 8 "up" outputs;
 //             out_bits[t][m] = round(silu(gate_m) * up_m) for the N/2 pairs m.
-// Each (token, output) is finished by exactly one thread of the cluster.  Every thread of
-// every block of the cluster must call this (it holds cluster barriers).
+// Block q of the cluster finishes the outputs (pairs) o with o % S == q: every block pushes
+// its partial sums into the owners' GemvRecv through distributed shared memory, one cluster
+// barrier later each owner adds the S contributions in rank order.  Every thread of every
+// block of the cluster must call this, after one cluster_arrive() earlier in the kernel.
 template <int DT, int TMAX, int PW, int CAP, int EP>
 __device__ __forceinline__ void gemv_finish_tile(float (&acc)[TMAX][8], int T, int tile,
-                                                 GemvSmem<TMAX, CAP>* sm, const EpilogueArgs& ep) {
+                                                 GemvSmem<TMAX, CAP>* sm, GemvRecv<TMAX>* recv,
+                                                 const EpilogueArgs& ep) {
     constexpr int LPC = PW / 8;
+    constexpr int HP = PW / 2;  // gate/up pairs per tile
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     cg::cluster_group cluster = cg::this_cluster();
     const int S = static_cast<int>(cluster.num_blocks());
     const int rank = static_cast<int>(cluster.block_rank());
+    const int W = EP == EP_SILU ? 2 * ((HP + S - 1) / S) : (PW + S - 1) / S;  // values per (source, token)
+    // where this thread's output goes: owner block and slot inside the owner's row
+    int owner = 0, slot = 0;
+    if (threadIdx.x < PW) {
+        const int o = threadIdx.x;
+        if (EP == EP_SILU) {
+            const int r = (o >> 4) * 8 + (o & 7);  // pair index; bit 3 of o says gate (0) / up (1)
+            owner = r % S;
+            slot = (r / S) * 2 + ((o >> 3) & 1);
+        } else {
+            owner = o % S;
+            slot = o / S;
+        }
+    }
+    float* dst = cluster.map_shared_rank(&recv->v[0], owner);
+    cluster_wait();  // pairs with the cluster_arrive() at kernel start: all peers are running
 #pragma unroll
     for (int t = 0; t < TMAX; ++t) {
         if (t < T) {
@@ -104,59 +142,50 @@ __device__ __forceinline__ void gemv_finish_tile(float (&acc)[TMAX][8], int T, i
                 for (int q = 0; q < 8; ++q) acc[t][q] += __shfl_xor_sync(0xFFFFFFFFu, acc[t][q], o);
             __syncthreads();
             if (lane < LPC) {
-                float4* dst = reinterpret_cast<float4*>(&sm->red[warp][lane * 8]);
-                dst[0] = make_float4(acc[t][0], acc[t][1], acc[t][2], acc[t][3]);
-                dst[1] = make_float4(acc[t][4], acc[t][5], acc[t][6], acc[t][7]);
+                float4* d4 = reinterpret_cast<float4*>(&sm->red[warp][lane * 8]);
+                d4[0] = make_float4(acc[t][0], acc[t][1], acc[t][2], acc[t][3]);
+                d4[1] = make_float4(acc[t][4], acc[t][5], acc[t][6], acc[t][7]);
             }
             __syncthreads();
             if (threadIdx.x < PW) {
                 float s = 0.0f;
 #pragma unroll
                 for (int g = 0; g < kGemvWarps; ++g) s += sm->red[g][threadIdx.x];
-                sm->part[t][threadIdx.x] = s;
+                dst[(rank * T + t) * W + slot] = s;
             }
         }
     }
-    cluster.sync();  // every block's part[][] is complete and visible
-    const float* parts[kMaxCluster];
-#pragma unroll
-    for (int q = 0; q < kMaxCluster; ++q)
-        parts[q] = q < S ? cluster.map_shared_rank(&sm->part[0][0], q) : nullptr;
+    cluster.sync();  // every contribution has landed
+    const float* mine = &recv->v[0];
     if (EP == EP_SILU) {
-        constexpr int HP = PW / 2;  // pairs per tile
-        const int total = T * HP;
-        for (int e = rank + S * static_cast<int>(threadIdx.x); e < total; e += S * kGemvThreads) {
-            const int t = e / HP, r = e - t * HP;
-            const int og = (r >> 3) * 16 + (r & 7);
+        const int WP = W / 2;
+        for (int e = threadIdx.x; e < T * WP; e += kGemvThreads) {
+            const int t = e / WP, ps = e - t * WP;
+            const int r = ps * S + rank;
             const int m = tile * HP + r;
-            if (2 * m < ep.N) {
+            if (r < HP && 2 * m < ep.N) {
                 float g = 0.0f, u = 0.0f;
-#pragma unroll
-                for (int q = 0; q < kMaxCluster; ++q)
-                    if (q < S) {
-                        g += parts[q][t * 256 + og];
-                        u += parts[q][t * 256 + og + 8];
-                    }
+                for (int q = 0; q < S; ++q) {
+                    g += mine[(q * T + t) * W + 2 * ps];
+                    u += mine[(q * T + t) * W + 2 * ps + 1];
+                }
                 const float v = g / (1.0f + expf(-g)) * u;
                 ep.out_bits[static_cast<size_t>(t) * (ep.N / 2) + m] = float_to_bits<DT>(v);
             }
         }
     } else {
-        const int total = T * PW;
-        for (int e = rank + S * static_cast<int>(threadIdx.x); e < total; e += S * kGemvThreads) {
-            const int t = e / PW, o = e - t * PW;
+        for (int e = threadIdx.x; e < T * W; e += kGemvThreads) {
+            const int t = e / W, sl = e - t * W;
+            const int o = sl * S + rank;
             const int out = tile * PW + o;
-            if (out < ep.N) {
+            if (o < PW && out < ep.N) {
                 float s = 0.0f;
-#pragma unroll
-                for (int q = 0; q < kMaxCluster; ++q)
-                    if (q < S) s += parts[q][t * 256 + o];
+                for (int q = 0; q < S; ++q) s += mine[(q * T + t) * W + sl];
                 float* p = ep.y + static_cast<size_t>(t) * ep.N + out;
                 *p = (EP == EP_ACCUM) ? *p + s : s;
             }
         }
     }
-    cluster.sync();  // nobody leaves while its shared memory may still be read
 }
 
 struct GemvListArgs {
@@ -173,12 +202,14 @@ struct GemvListArgs {
 
 // grid = (S, tiles), cluster = (S, 1, 1).
 template <int DT, int TMAX, int PW, int CAP>
-__device__ __forceinline__ void gemv_list_block(const GemvListArgs& a, GemvSmem<TMAX, CAP>* sm) {
+__device__ __forceinline__ void gemv_list_block(const GemvListArgs& a, GemvSmem<TMAX, CAP>* sm,
+                                                GemvRecv<TMAX>* recv) {
     constexpr int LPC = PW / 8;
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int S = gridDim.x, s = blockIdx.x, tile = blockIdx.y;
     const int T = a.T;
+    cluster_arrive();
     // Programmatic dependent launch: let the next grid in the stream be scheduled as soon as
     // SM resources free up, and touch global memory only once the previous grid is complete.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -210,9 +241,9 @@ __device__ __forceinline__ void gemv_list_block(const GemvListArgs& a, GemvSmem<
         if (lane_ok) gemv_stream<DT, TMAX, PW, CAP>(a.Wt + out0, a.ldw, T, sm, staged, acc);
     }
     if (a.accumulate)
-        gemv_finish_tile<DT, TMAX, PW, CAP, EP_ACCUM>(acc, T, tile, sm, a.ep);
+        gemv_finish_tile<DT, TMAX, PW, CAP, EP_ACCUM>(acc, T, tile, sm, recv, a.ep);
     else
-        gemv_finish_tile<DT, TMAX, PW, CAP, EP_STORE>(acc, T, tile, sm, a.ep);
+        gemv_finish_tile<DT, TMAX, PW, CAP, EP_STORE>(acc, T, tile, sm, recv, a.ep);
 }
 
 }  // namespace afx

@@ -21,7 +21,8 @@ fused_op_kernel(FusedArgs a) {
     constexpr int CAP = FusedShape<TMAX>::kStageCap;
     extern __shared__ __align__(16) unsigned char dyn[];
     __shared__ SelectScratch sel;
-    fused_op_block<DT, TMAX, PW, CAP, IN, EP>(a, dyn, &sel);
+    __shared__ GemvRecv<TMAX> recv;
+    fused_op_block<DT, TMAX, PW, CAP, IN, EP>(a, dyn, &sel, &recv);
 }
 
 template <int DT, int REP>
