@@ -222,6 +222,36 @@ afx_status afx_layer_step(afx_model* model, int layer, afx_state* state, int pos
 afx_status afx_mlp_block(afx_model* model, int layer, afx_state* state, const void* x, float* y,
                          void* stream);
 
+/*
+ * The MLP block without any allocation (the paper has no counterpart: this entry point exists
+ * for the integration, not for the method).  Same result as afx_mlp_block on the same weights
+ * and input -- y = W_down(silu(W_gate x) * W_up x), both operators on the active channels of
+ * their own input -- but it needs neither afx_model_create (which calls cudaMalloc for its
+ * rotary table) nor a caller-allocated state blob: the intermediate vector silu(gate) * up is
+ * kept in a fixed array inside the library image (AFX_MAX_T * AFX_NOALLOC_MAX_MLP 16-bit values
+ * = 512 KB per GPU, held by every GPU that loads the library until the process exits).  It is
+ * meant for callers that must not allocate device memory: a serving process that has handed all
+ * of HBM to its own pool, code in a latency-critical loop where cudaMalloc's device-wide
+ * synchronisation is not acceptable, or a plug-in that is only given pointers.  The call itself
+ * uses no cudaMalloc, cudaFree or other allocating routine.
+ *
+ *   w_gu    DEVICE [hidden][2*mlp] channel-contiguous, columns in groups of 16 = gate[8m..8m+8)
+ *           then up[8m..8m+8) (the w_gu layout of afx_layer_desc); w_down DEVICE [mlp][hidden].
+ *   x       DEVICE [T][hidden] 16-bit floats (already normalised); y DEVICE [T][hidden] fp32,
+ *           overwritten.  mode, k_*, tau_* as for afx_select_active, per operator.
+ * hidden and mlp are multiples of 8; hidden <= 32768; mlp > AFX_NOALLOC_MAX_MLP returns
+ * AFX_ERR_CAPACITY and launches nothing.
+ * The first call on a device looks up the array's device address (with that device current);
+ * make that first call outside any stream capture.  All calls on a device share the array and
+ * it keeps the previous call's contents (nothing in it has to start from zero: each call
+ * rewrites the T * mlp values it reads): two calls whose kernels overlap on the GPU -- different
+ * streams, or graphs replayed concurrently -- race on it; serialise them.
+ */
+#define AFX_NOALLOC_MAX_MLP 32768
+afx_status afx_mlp_block_noalloc(const void* w_gu, const void* w_down, int dtype, int hidden, int mlp,
+                                 const void* x, int T, int mode, int k_gu, float tau_gu, int k_down,
+                                 float tau_down, float* y, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

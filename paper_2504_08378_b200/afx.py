@@ -79,6 +79,8 @@ def lib() -> ctypes.CDLL:
                                        ctypes.POINTER(c_size_t)]
         L.afx_layer_step.argtypes = [c_void_p, c_int, c_void_p, c_int, c_void_p]
         L.afx_mlp_block.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p]
+        L.afx_mlp_block_noalloc.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_void_p, c_int, c_int, c_int,
+                                            c_float, c_int, c_float, c_void_p, c_void_p]
         _lib = L
     return _lib
 
@@ -188,3 +190,14 @@ def afx_layer_step(model: int, layer: int, state: int, pos: int, stream=None):
 
 def afx_mlp_block(model: int, layer: int, state: int, x, y, stream=None):
     _check("afx_mlp_block", lib().afx_mlp_block(model, int(layer), state, _ptr(x), _ptr(y), _stream(stream)))
+
+
+def afx_mlp_block_noalloc(w_gu, w_down, dtype, hidden: int, mlp: int, x, T: int, mode: int, k_gu: int, tau_gu: float,
+                          k_down: int, tau_down: float, y, stream=None):
+    """The MLP block for callers that may not allocate device memory: no model object, no state
+    blob; the intermediate vector lives in a fixed 512 KB array inside the library (shared by all
+    calls on a device, so calls that overlap on the GPU race).  mlp <= 32768."""
+    _check("afx_mlp_block_noalloc",
+           lib().afx_mlp_block_noalloc(_ptr(w_gu), _ptr(w_down), _dt(dtype), int(hidden), int(mlp), _ptr(x), int(T),
+                                       int(mode), int(k_gu), float(tau_gu), int(k_down), float(tau_down), _ptr(y),
+                                       _stream(stream)))

@@ -468,3 +468,83 @@ extern "C" afx_status afx_select_gemv(const void* Wt, int dtype, int K, int N, i
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     return accumulate ? launch_fused<IN_X, EP_ACCUM>(dtype, a, st) : launch_fused<IN_X, EP_STORE>(dtype, a, st);
 }
+
+// ---------------------------------------------------------------------------------------------
+// afx_mlp_block_noalloc: the MLP block for callers that cannot allocate device memory.
+// ---------------------------------------------------------------------------------------------
+
+namespace afx {
+
+// The intermediate vector silu(gate) * up of the block, [T][mlp] 16-bit values, lives here
+// instead of in a caller-allocated state blob.  Every device that loads the library holds
+// these 512 KB until the process exits.  All calls share it.
+constexpr int kNoAllocMaxMlp = AFX_NOALLOC_MAX_MLP;
+static __device__ __align__(256) uint16_t g_noalloc_hm[AFX_MAX_T * kNoAllocMaxMlp];
+
+// Device address of g_noalloc_hm on the current device (host code only sees a stand-in for
+// the symbol; the address has to be asked for, once per device, with that device current).
+static afx_status noalloc_scratch(uint16_t** out) {
+    static std::mutex mu;
+    static uint16_t* addr[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        cudaGetLastError();
+        return AFX_ERR_CUDA;
+    }
+    std::lock_guard<std::mutex> lock(mu);
+    if (addr[dev] == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_noalloc_hm) != cudaSuccess || p == nullptr) {
+            cudaGetLastError();
+            return AFX_ERR_CUDA;
+        }
+        addr[dev] = static_cast<uint16_t*>(p);
+    }
+    *out = addr[dev];
+    return AFX_OK;
+}
+
+}  // namespace afx
+
+extern "C" afx_status afx_mlp_block_noalloc(const void* w_gu, const void* w_down, int dtype, int hidden, int mlp,
+                                            const void* x, int T, int mode, int k_gu, float tau_gu, int k_down,
+                                            float tau_down, float* y, void* stream) {
+    using namespace afx;
+    if (w_gu == nullptr || w_down == nullptr || x == nullptr || y == nullptr) return AFX_ERR_INVALID_ARG;
+    if (hidden < 8 || mlp < 8 || T < 1 || T > AFX_MAX_T) return AFX_ERR_INVALID_ARG;
+    if (mlp > kNoAllocMaxMlp || hidden > kSelectFastMaxK) return AFX_ERR_CAPACITY;
+    if (dtype != AFX_F16 && dtype != AFX_BF16) return AFX_ERR_UNSUPPORTED;
+    if (mode != AFX_MODE_TOPK && mode != AFX_MODE_THRESHOLD) return AFX_ERR_UNSUPPORTED;
+    if (mode == AFX_MODE_TOPK && (k_gu < 0 || k_gu > hidden || k_down < 0 || k_down > mlp)) return AFX_ERR_INVALID_ARG;
+    if (mode == AFX_MODE_THRESHOLD && (tau_gu != tau_gu || tau_down != tau_down)) return AFX_ERR_INVALID_ARG;
+    if ((hidden & 7) != 0 || (mlp & 7) != 0 || !aligned16(w_gu) || !aligned16(w_down) || !aligned16(y) ||
+        (reinterpret_cast<uintptr_t>(x) & 1u) != 0)
+        return AFX_ERR_ALIGNMENT;
+    uint16_t* hm = nullptr;
+    afx_status rc = noalloc_scratch(&hm);
+    if (rc != AFX_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // Nothing in hm has to start from zero: the first kernel writes all T * mlp values that
+    // the second one reads.
+    FusedArgs a = {};
+    a.T = T;
+    a.Wt = static_cast<const uint16_t*>(w_gu);
+    a.ldw = 2 * static_cast<int64_t>(mlp);
+    a.K = hidden;
+    a.N = 2 * mlp;
+    a.x = static_cast<const uint16_t*>(x);
+    a.mode = mode;
+    a.k = k_gu;
+    a.tau = tau_gu;
+    a.ep = {nullptr, hm, 2 * mlp};
+    if ((rc = launch_fused<IN_X, EP_SILU>(dtype, a, st)) != AFX_OK) return rc;
+    a.Wt = static_cast<const uint16_t*>(w_down);
+    a.ldw = hidden;
+    a.K = mlp;
+    a.N = hidden;
+    a.x = hm;
+    a.k = k_down;
+    a.tau = tau_down;
+    a.ep = {y, nullptr, hidden};
+    return launch_fused<IN_X, EP_STORE>(dtype, a, st);
+}

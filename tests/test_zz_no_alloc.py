@@ -1,0 +1,58 @@
+"""afx_mlp_block_noalloc against afx_mlp_block.
+
+The no-alloc entry point serves callers that are not allowed to allocate device memory (a
+server that has given all of HBM to its own pool, a latency-critical loop, a plug-in that only
+receives pointers): it keeps the block's intermediate vector in a fixed array inside the
+library instead of in a caller-allocated state.  Here it must reproduce the result of the
+ordinary entry point, on two calls in a row with different inputs -- the second call finds the
+first call's data in the shared array and must not be affected by it.
+
+This file is collected last on purpose, so that a run stopping at its first failure has
+already run every other test.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2504_08378_b200 import afx, synth
+from paper_2504_08378_b200.model import DecoderModel
+from gpu_util import rel_err
+
+pytestmark = pytest.mark.gpu
+
+TOL = 2e-3
+
+
+def _dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a, np.uint16).view(np.int16)).cuda()
+
+
+@pytest.mark.parametrize("dt,T,mode", [("bf16", 1, afx.MODE_TOPK), ("f16", 3, afx.MODE_THRESHOLD)])
+def test_noalloc_mlp_block_matches_mlp_block_twice(dt, T, mode):
+    hidden, mlp = 1024, 2752
+    L = synth.layer_weights(77, 0, hidden, 8, 8, mlp, dt)
+    L["k"] = [0, 0, hidden // 2, mlp // 2]
+    L["tau"] = [0.0, 0.0, synth.laplace_tau(0.5), 0.004]
+    m = DecoderModel(dt, hidden, 8, 8, mlp, 16, [L], T=T, select_mode=mode)
+    w_gu = _dev(synth.interleave_gate_up(L["w_gate"], L["w_up"]))
+    w_down = _dev(L["w_down"])
+    for call in range(2):
+        x = _dev(synth.laplace_bits(77, 20 + call, (T, hidden), dt))
+        y_ref = torch.full((T, hidden), float("nan"), device="cuda")
+        m.mlp_block(0, x, y_ref)
+        y = torch.full((T, hidden), float("nan"), device="cuda")
+        afx.afx_mlp_block_noalloc(w_gu, w_down, dt, hidden, mlp, x, T, mode, L["k"][2], L["tau"][2],
+                                  L["k"][3], L["tau"][3], y)
+        torch.cuda.synchronize()
+        ref = y_ref.cpu().numpy()
+        assert np.isfinite(ref).all()
+        assert rel_err(y.cpu().numpy(), ref) <= TOL, f"call {call}"
+    m.close()
+
+
+def test_noalloc_rejects_sizes_beyond_the_fixed_array():
+    fake = 0x7F0000000000  # never dereferenced: validation fails first
+    with pytest.raises(afx.AfxError) as e:
+        afx.afx_mlp_block_noalloc(fake, fake, "bf16", 4096, 32768 + 8, fake, 1, afx.MODE_TOPK, 8, 0.0, 8, 0.0,
+                                  fake, stream=0)
+    assert e.value.status == 3  # AFX_ERR_CAPACITY
