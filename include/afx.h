@@ -222,6 +222,74 @@ afx_status afx_layer_step(afx_model* model, int layer, afx_state* state, int pos
 afx_status afx_mlp_block(afx_model* model, int layer, afx_state* state, const void* x, float* y,
                          void* stream);
 
+/* ------------------------------------------------------------------------------------------
+ * Hot-weight cache (Sec. 4.2 "Dynamic LLM Weight Caching": per weight tensor a table from
+ * channel to cache slot and a usage count per channel that starts from zero with every new
+ * sequence; a newly active channel replaces the least used cached one).  The full operator
+ * lives in pinned HOST memory (standing in for flash); the cache holds `capacity` of its
+ * channels in DEVICE memory.  afx_cache_fetch takes one step's active list, counts the usage,
+ * decides hits / replacements, copies every missed channel from the host into its slot and
+ * returns the slot of each active channel, which afx_sparse_gemv accepts as its `slot` list.
+ *
+ * Policy, for the ascending active list of one step:
+ *   1. count[j] += 1 for every active j;  2. a channel that already has a slot is a hit;
+ *   3. misses in ascending channel order: the lowest free slot if there is one; otherwise the
+ *      cached channel that is NOT active in this step with the smallest (count, channel id) is
+ *      the victim and is replaced when count[miss] >= count[victim] (the paper's worked example
+ *      replaces on equal counts); a miss that replaces nothing is "transient": it is copied
+ *      into staging row capacity + r (r = its rank among this step's transients), used for
+ *      this step and not retained.
+ * ------------------------------------------------------------------------------------------ */
+
+typedef struct afx_cache afx_cache; /* opaque, HOST object owning small DEVICE tables */
+
+typedef struct {
+    int32_t dtype;         /* AFX_F16 / AFX_BF16                                                 */
+    int32_t K, N;          /* channels of the operator, values per channel (N % 8 == 0)          */
+    int64_t ldw;           /* row stride in elements of BOTH host_base and slots (ldw % 8 == 0)  */
+    int32_t capacity;      /* cached channels C, 1 <= C <= K                                     */
+    int32_t staging_rows;  /* rows after the C cache rows for transient channels (>= 0)          */
+    const void* host_base; /* HOST, [K][ldw], page-locked (cudaHostAlloc / cudaHostRegister)     */
+    void* slots;           /* DEVICE, [C + staging_rows][ldw], 16-byte aligned, caller-owned     */
+} afx_cache_desc;
+
+typedef struct {
+    int32_t hits, misses, transients; /* of the last afx_cache_fetch                            */
+    int32_t overflow;                 /* transients that did not fit into staging_rows (their   */
+                                      /* slot is -1: the step's result must not be used)        */
+    uint64_t bytes_fetched;           /* host -> device bytes of the last fetch: copied * N * 2 */
+} afx_cache_stats;
+
+/*
+ * afx_cache_create checks the descriptor, resolves the device view of host_base (returns
+ * AFX_ERR_INVALID_ARG when it is not page-locked) and allocates the tables (cudaMalloc:
+ * slot per channel, channel per slot, count per channel, work lists; about 24 bytes per
+ * channel).  The cache starts empty.  afx_cache_destroy frees them.
+ */
+afx_status afx_cache_create(const afx_cache_desc* desc, afx_cache** out);
+afx_status afx_cache_destroy(afx_cache* cache);
+
+/* New sequence: every usage count returns to zero; cached channels stay.  Enqueued on stream. */
+afx_status afx_cache_reset(afx_cache* cache, void* stream);
+
+/* Pre-load channels (HOST list, n <= free slots, not yet cached) into the lowest free slots,
+ * copying their columns; used to set the initial cache contents.  Synchronises the stream. */
+afx_status afx_cache_install(afx_cache* cache, const int32_t* host_channels, int n, void* stream);
+
+/*
+ * One step.  idx / count: DEVICE active list (ascending; as afx_select_active writes it).
+ * slot_out: DEVICE int32[K]; entry c receives the row of idx[c] in `slots`.  stats: DEVICE
+ * afx_cache_stats or NULL.  Two kernels on `stream`: the policy (one thread block; the
+ * victims are ordered by a bitonic sort of (count, channel) keys) and the copy of the missed
+ * channels (128-bit loads from the mapped host memory).  No host synchronisation.
+ */
+afx_status afx_cache_fetch(afx_cache* cache, const int32_t* idx, const int32_t* count, int32_t* slot_out,
+                           afx_cache_stats* stats, void* stream);
+
+/* Copies the tables to HOST arrays for inspection (either may be NULL): slot_of[K] (-1 = not
+ * cached), usage[K].  Synchronises the stream. */
+afx_status afx_cache_snapshot(afx_cache* cache, int32_t* host_slot_of, uint32_t* host_usage, void* stream);
+
 /*
  * The MLP block without any allocation (the paper has no counterpart: this entry point exists
  * for the integration, not for the method).  Same result as afx_mlp_block on the same weights

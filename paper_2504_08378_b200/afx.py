@@ -41,6 +41,18 @@ class LayerDesc(ctypes.Structure):
                 ("k", c_int32 * 4), ("tau", c_float * 4)]
 
 
+class CacheDesc(ctypes.Structure):
+    """afx_cache_desc"""
+    _fields_ = [("dtype", c_int32), ("K", c_int32), ("N", c_int32), ("ldw", c_int64), ("capacity", c_int32),
+                ("staging_rows", c_int32), ("host_base", c_void_p), ("slots", c_void_p)]
+
+
+class CacheStats(ctypes.Structure):
+    """afx_cache_stats"""
+    _fields_ = [("hits", c_int32), ("misses", c_int32), ("transients", c_int32), ("overflow", c_int32),
+                ("bytes_fetched", ctypes.c_uint64)]
+
+
 class AfxError(RuntimeError):
     def __init__(self, fn: str, status: int):
         self.status = status
@@ -79,6 +91,12 @@ def lib() -> ctypes.CDLL:
                                        ctypes.POINTER(c_size_t)]
         L.afx_layer_step.argtypes = [c_void_p, c_int, c_void_p, c_int, c_void_p]
         L.afx_mlp_block.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p]
+        L.afx_cache_create.argtypes = [ctypes.POINTER(CacheDesc), ctypes.POINTER(c_void_p)]
+        L.afx_cache_destroy.argtypes = [c_void_p]
+        L.afx_cache_reset.argtypes = [c_void_p, c_void_p]
+        L.afx_cache_install.argtypes = [c_void_p, c_void_p, c_int, c_void_p]
+        L.afx_cache_fetch.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+        L.afx_cache_snapshot.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p]
         L.afx_mlp_block_noalloc.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_void_p, c_int, c_int, c_int,
                                             c_float, c_int, c_float, c_void_p, c_void_p]
         _lib = L
@@ -201,3 +219,38 @@ def afx_mlp_block_noalloc(w_gu, w_down, dtype, hidden: int, mlp: int, x, T: int,
            lib().afx_mlp_block_noalloc(_ptr(w_gu), _ptr(w_down), _dt(dtype), int(hidden), int(mlp), _ptr(x), int(T),
                                        int(mode), int(k_gu), float(tau_gu), int(k_down), float(tau_down), _ptr(y),
                                        _stream(stream)))
+
+
+def afx_cache_create(desc: CacheDesc) -> int:
+    out = c_void_p(0)
+    _check("afx_cache_create", lib().afx_cache_create(ctypes.byref(desc), ctypes.byref(out)))
+    return out.value
+
+
+def afx_cache_destroy(cache: int):
+    _check("afx_cache_destroy", lib().afx_cache_destroy(cache))
+
+
+def afx_cache_reset(cache: int, stream=None):
+    _check("afx_cache_reset", lib().afx_cache_reset(cache, _stream(stream)))
+
+
+def afx_cache_install(cache: int, channels, stream=None):
+    """channels: sequence of channel ids (host side) pre-loaded into the lowest free slots."""
+    arr = (c_int32 * len(channels))(*[int(c) for c in channels])
+    _check("afx_cache_install", lib().afx_cache_install(cache, arr, len(channels), _stream(stream)))
+
+
+def afx_cache_fetch(cache: int, idx, count, slot_out, stats=None, stream=None):
+    _check("afx_cache_fetch",
+           lib().afx_cache_fetch(cache, _ptr(idx), _ptr(count), _ptr(slot_out), _ptr(stats), _stream(stream)))
+
+
+def afx_cache_snapshot(cache: int, K: int, stream=None):
+    """Returns (slot_of[K] int32, usage[K] uint32) as numpy arrays."""
+    import numpy as np
+    slot_of = np.empty(K, np.int32)
+    usage = np.empty(K, np.uint32)
+    _check("afx_cache_snapshot",
+           lib().afx_cache_snapshot(cache, slot_of.ctypes.data, usage.ctypes.data, _stream(stream)))
+    return slot_of, usage
