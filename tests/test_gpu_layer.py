@@ -20,9 +20,17 @@ def bits_np(t):
     return t.cpu().numpy().view(np.uint16)
 
 
-def ulp_close(a, b, frac_exact=0.98):
+def ulp_close(a, b, frac_exact=0.98, dt=None):
+    """16-bit results of the same arithmetic in fp32 (GPU) and fp64 (oracle): nearly all bit
+    patterns equal, the rest one step apart -- or, where a value sits next to zero after
+    cancellation (its last place is then far below the sum's own rounding error), within
+    1e-3 of the vector's rms (needs dt to decode)."""
     d = np.abs(a.astype(np.int32) - b.astype(np.int32))
-    return (d <= 1).all() and (d == 0).mean() >= frac_exact
+    ok = d <= 1
+    if dt is not None and not ok.all():
+        va, vb = oracle.decode(a, dt), oracle.decode(b, dt)
+        ok |= np.abs(va - vb) <= 1e-3 * np.sqrt(np.mean(vb ** 2))
+    return ok.all() and (d == 0).mean() >= frac_exact
 
 
 def make(cfg, layers_np, T, mode, xl_depth=0, xl_mode=0, max_seq=64):
@@ -66,13 +74,13 @@ def check_layer_stages(cfg, L, lw, m, layer, h0, kc0, vc0, pos, T):
     h1_ref = h0.astype(np.float64) + oracle.sparse_gemv(L["w_o"], dt, cfg.hidden, attn_gpu, idx_o)
     # gate/up
     xm_gpu = bits_np(m.bits(afx.BUF_XNORM, afx.OP_GU))
-    assert ulp_close(xm_gpu, oracle.rmsnorm(h1_ref, lw.g_mlp, cfg.eps, dt), frac_exact=0.97)
+    assert ulp_close(xm_gpu, oracle.rmsnorm(h1_ref, lw.g_mlp, cfg.eps, dt), frac_exact=0.97, dt=dt)
     idx_gu = m.idx(afx.OP_GU).cpu().numpy()[: stats[2][0]]
     assert np.array_equal(idx_gu, ol.select(xm_gpu, cfg, lw, "gu"))
     g = oracle.sparse_gemv(L["w_gate"], dt, cfg.mlp, xm_gpu, idx_gu)
     u = oracle.sparse_gemv(L["w_up"], dt, cfg.mlp, xm_gpu, idx_gu)
     hm_gpu = bits_np(m.bits(afx.BUF_HM))
-    assert ulp_close(hm_gpu, oracle.silu_mul(g, u, dt), frac_exact=0.97)
+    assert ulp_close(hm_gpu, oracle.silu_mul(g, u, dt), frac_exact=0.97, dt=dt)
     # down
     idx_d = m.idx(afx.OP_DOWN).cpu().numpy()[: stats[3][0]]
     assert np.array_equal(idx_d, ol.select(hm_gpu, cfg, lw, "down"))
