@@ -147,15 +147,35 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
     int cnt = 0;
     int pos0 = 0;                  // list position of this thread's first active channel
     unsigned long long fl = 0ull;  // this thread's active flags (own selection)
+    const int out0 = tile * PW + (lane % LPC) * 8;
+    const bool lane_ok = out0 < a.N;
+    // One token, top-k: the list length is k whatever x holds, so this block's part
+    // [c_lo, c_hi) of the list is known before the selection and the pass that decides the
+    // flags (it has the channel's bits in registers) stages the first CAP entries directly.
+    const bool early = topk && T == 1;
+    bool first_staged = false;
     if (own) {
+        const int e_lo = s * a.k / S, e_n = min(CAP, (s + 1) * a.k / S - e_lo);
         for (int t = 0; t < T; ++t) {
             const uint16_t* xt = xs + (IN == IN_NORM ? static_cast<size_t>(t) * Kp : 0);
             if (IN == IN_X) {
                 if (t > 0) __syncthreads();  // the previous token's keys are still being read
                 block_stage_token(a.x + static_cast<size_t>(t) * K, K, xs);
             }
-            fl |= block_token_flags<DT, kGemvThreads>(xt, K, a.mode, a.k, a.tau, hist, t == 0, sel, T == 1,
-                                                      pos0, cnt);
+            if (early) {
+                fl |= block_token_flags<DT, kGemvThreads>(
+                    xt, K, a.mode, a.k, a.tau, hist, t == 0, sel, true, pos0, cnt, [&](int j, int pos, uint16_t bits) {
+                        const int p = pos - e_lo;
+                        if (p >= 0 && p < e_n) {  // the histogram is dead by now: its memory is the staging area
+                            sm->col[p] = j;
+                            sm->xv[0][p] = bits_to_float<DT>(bits);
+                        }
+                    });
+                first_staged = true;
+            } else {
+                fl |= block_token_flags<DT, kGemvThreads>(xt, K, a.mode, a.k, a.tau, hist, t == 0, sel, T == 1,
+                                                          pos0, cnt);
+            }
         }
         if (T > 1) pos0 = block_prefix(__popcll(fl), sel->wtot[2], cnt);
         if (scribe) store_flag_bytes(fl, K, flags);
@@ -167,8 +187,6 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
     AFX_MARK(3);
     const int c_lo = s * cnt / S;  // S <= 8, cnt <= 2^20: no overflow
     const int c_hi = (s + 1) * cnt / S;
-    const int out0 = tile * PW + (lane % LPC) * 8;
-    const bool lane_ok = out0 < a.N;
 
     float acc[TMAX][8];
 #pragma unroll
@@ -176,27 +194,32 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
 #pragma unroll
         for (int q = 0; q < 8; ++q) acc[t][q] = 0.0f;
 
+    const int n_mine = __popcll(fl);
     for (int c0 = c_lo; c0 < c_hi; c0 += CAP) {
         const int staged = min(CAP, c_hi - c0);
-        __syncthreads();  // the work area is free: the histogram / the previous stage has been read
-        // ---- stage (column, x values) of list positions [c0, c0 + staged) ----
-        if (own) {
-            for_each_owned_active(fl, K, pos0, [&](int j, int pos) {
-                const int p = pos - c0;
-                if (p >= 0 && p < staged) {
-                    sm->col[p] = j;
+        if (!(first_staged && c0 == c_lo)) {
+            __syncthreads();  // the work area is free: the histogram / the previous stage has been read
+            // ---- stage (column, x values) of list positions [c0, c0 + staged) ----
+            if (own) {
+                if (pos0 < c0 + staged && pos0 + n_mine > c0) {
+                    for_each_owned_active(fl, K, pos0, [&](int j, int pos) {
+                        const int p = pos - c0;
+                        if (p >= 0 && p < staged) {
+                            sm->col[p] = j;
+#pragma unroll
+                            for (int t = 0; t < TMAX; ++t)
+                                if (t < T) sm->xv[t][p] = bits_to_float<DT>(x_at(t, j));
+                        }
+                    });
+                }
+            } else {
+                for (int i = tid; i < staged; i += kGemvThreads) {
+                    const int j = a.idx_in[c0 + i];
+                    sm->col[i] = j;
 #pragma unroll
                     for (int t = 0; t < TMAX; ++t)
-                        if (t < T) sm->xv[t][p] = bits_to_float<DT>(x_at(t, j));
+                        if (t < T) sm->xv[t][i] = bits_to_float<DT>(x_at(t, j));
                 }
-            });
-        } else {
-            for (int i = tid; i < staged; i += kGemvThreads) {
-                const int j = a.idx_in[c0 + i];
-                sm->col[i] = j;
-#pragma unroll
-                for (int t = 0; t < TMAX; ++t)
-                    if (t < T) sm->xv[t][i] = bits_to_float<DT>(x_at(t, j));
             }
         }
         __syncthreads();

@@ -104,11 +104,12 @@ __device__ __forceinline__ void gemv_stream(const uint16_t* __restrict__ wbase, 
 // Block q of the cluster finishes the outputs (pairs) o with o % S == q: every block pushes
 // its partial sums into the owners' GemvRecv through distributed shared memory, one cluster
 // barrier later each owner adds the S contributions in rank order.  Every thread of every
-// block of the cluster must call this, after one cluster_arrive() earlier in the kernel.
+// block of the cluster must call this, after one cluster_arrive() earlier in the kernel whose
+// wait is still pending (pending_wait) or has been taken by the caller since.
 template <int DT, int TMAX, int PW, int CAP, int EP>
 __device__ __forceinline__ void gemv_finish_tile(float (&acc)[TMAX][8], int T, int tile,
                                                  GemvSmem<TMAX, CAP>* sm, GemvRecv<TMAX>* recv,
-                                                 const EpilogueArgs& ep) {
+                                                 const EpilogueArgs& ep, bool pending_wait = true) {
     constexpr int LPC = PW / 8;
     constexpr int HP = PW / 2;  // gate/up pairs per tile
     const int lane = threadIdx.x & 31;
@@ -131,7 +132,7 @@ __device__ __forceinline__ void gemv_finish_tile(float (&acc)[TMAX][8], int T, i
         }
     }
     float* dst = cluster.map_shared_rank(&recv->v[0], owner);
-    cluster_wait();  // pairs with the cluster_arrive() at kernel start: all peers are running
+    if (pending_wait) cluster_wait();  // pairs with the cluster_arrive() at kernel start: all peers are running
 #pragma unroll
     for (int t = 0; t < TMAX; ++t) {
         if (t < T) {

@@ -12,7 +12,7 @@ namespace afx {
 template <int TMAX>
 struct FusedShape {
     static constexpr int kBlocksPerSM = TMAX <= 1 ? 2 : 1;
-    static constexpr int kStageCap = TMAX <= 4 ? 1024 : 512;
+    static constexpr int kStageCap = TMAX <= 4 ? 2048 : 1024;
 };
 
 template <int DT, int TMAX, int PW, int IN, int EP>

@@ -200,12 +200,17 @@ __device__ __forceinline__ void block_kth_key(const uint16_t* xs, int K, int k, 
 // block_kth_key.  `hist` is the key histogram (top-k only); `hist_clean` says that it is
 // already zero and visible.  With `single` set (the token is the only one) the call also
 // returns the list position of the thread's first active channel in `pos0` and the length
-// of the list in `cnt`, from the same scan that orders the tie-break.
-template <int DT, int NT>
+// of the list in `cnt`, from the same scan that orders the tie-break, and calls
+// emit(channel, list position, 16-bit pattern) for every active channel of the thread.
+struct NoEmit {
+    __device__ __forceinline__ void operator()(int, int, uint16_t) const {}
+};
+
+template <int DT, int NT, class Emit = NoEmit>
 __device__ __forceinline__ unsigned long long block_token_flags(const uint16_t* xs, int K, int mode, int k,
                                                                 float tau, uint32_t* hist, bool hist_clean,
                                                                 SelectScratch* s, bool single, int& pos0,
-                                                                int& cnt) {
+                                                                int& cnt, Emit emit = Emit()) {
     int c_lo, c_hi;
     thread_chunk_range(K, c_lo, c_hi);
     unsigned long long fl = 0ull;
@@ -225,7 +230,14 @@ __device__ __forceinline__ unsigned long long block_token_flags(const uint16_t* 
             }
             fl |= static_cast<unsigned long long>(byte) << (8 * (c - c_lo));
         }
-        if (single) pos0 = block_prefix(__popcll(fl), s->wtot[1], cnt);
+        if (single) {
+            pos0 = block_prefix(__popcll(fl), s->wtot[1], cnt);
+            int pos = pos0;
+            for (unsigned long long rest = fl; rest != 0ull; rest &= rest - 1ull) {
+                const int j = (c_lo << 3) + __ffsll(static_cast<long long>(rest)) - 1;
+                emit(j, pos++, xs[j]);
+            }
+        }
         return fl;
     }
     if (!hist_clean) {
@@ -259,17 +271,21 @@ __device__ __forceinline__ unsigned long long block_token_flags(const uint16_t* 
         pre_e = block_prefix(e_cnt, s->wtot[1], tot);
     }
     int seen_e = pre_e;
+    int pos = pos0;
     for (int c = c_lo; c < c_hi; ++c) {
-        uint32_t key[8];
-        chunk_keys(xs, c, key);
+        const uint4 raw = *reinterpret_cast<const uint4*>(xs + (c << 3));
+        const uint32_t r[4] = {raw.x, raw.y, raw.z, raw.w};
         uint32_t byte = 0;
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
+            const uint32_t bits = (r[e >> 1] >> (16 * (e & 1))) & 0xFFFFu;
+            const uint32_t key = bits & 0x7FFFu;
             const bool in = (c << 3) + e < K;
-            const bool eq = in && key[e] == thr;
-            const bool pred = in && (key[e] > thr || (eq && (need_eq == tot_eq || seen_e < need_eq)));
+            const bool eq = in && key == thr;
+            const bool pred = in && (key > thr || (eq && (need_eq == tot_eq || seen_e < need_eq)));
             seen_e += eq;
             byte |= static_cast<uint32_t>(pred) << e;
+            if (single && pred) emit((c << 3) + e, pos++, static_cast<uint16_t>(bits));
         }
         fl |= static_cast<unsigned long long>(byte) << (8 * (c - c_lo));
     }

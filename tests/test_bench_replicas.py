@@ -19,20 +19,21 @@ WORKER = textwrap.dedent("""
     ms = bench.reduce_max_ms(10.0 * (rank + 1), world, backend_device="cpu")   # rank 1 is the slow replica
     steps = 5
     value = world * steps / (ms * 1e-3)                                         # whole-job tokens/s
-    print(json.dumps({{"rank": rank, "ms": ms, "value": value}}), flush=True)
+    with open(os.path.join({out!r}, f"rank{{rank}}.json"), "w") as f:           # one file per rank: stdout interleaves
+        json.dump({{"rank": rank, "ms": ms, "value": value}}, f)
     dist.destroy_process_group()
 """)
 
 
 def test_two_gloo_ranks_take_the_max_duration(tmp_path):
     script = tmp_path / "worker.py"
-    script.write_text(WORKER.format(root=ROOT))
+    script.write_text(WORKER.format(root=ROOT, out=str(tmp_path)))
     env = dict(os.environ, MASTER_ADDR="127.0.0.1", OMP_NUM_THREADS="1")
     out = subprocess.run([sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2",
                           "--master-addr", "127.0.0.1", "--master-port", "29631", str(script)],
                          capture_output=True, text=True, timeout=240, env=env, cwd=ROOT)
     assert out.returncode == 0, out.stderr[-2000:]
-    rows = [json.loads(l) for l in out.stdout.splitlines() if l.startswith("{")]
+    rows = [json.load(open(tmp_path / f"rank{r}.json")) for r in (0, 1)]
     assert sorted(r["rank"] for r in rows) == [0, 1]
     for r in rows:
         assert r["ms"] == 20.0                      # the slower replica's time on every rank
