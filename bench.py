@@ -142,6 +142,80 @@ def build_model(cfg):
     return m, layers, k
 
 
+def run_variants(cfg, layers, k, h0_dev, pos, st, steps):
+    """The same token in the method's two other documented forms (extra information, not the
+    headline): per-operator magnitude THRESHOLDS calibrated beforehand on other tokens instead
+    of exact top-k (the paper's own run-time form), and cross-layer REUSE (layers 3g+1..3g+3
+    compute on the set that layer 3g selected, no selection of their own)."""
+    import numpy as np
+    import torch
+    from paper_2504_08378_b200 import afx, synth
+    from paper_2504_08378_b200.model import DecoderModel
+    H, M, NL = cfg["hidden"], cfg["mlp"], cfg["n_layers"]
+    max_seq = cfg["past"] + 8
+    K_op = (H, cfg["n_heads"] * 128, H, M)
+
+    def model(layer_dicts, mode, xl_mode):
+        return DecoderModel(cfg["dtype"], H, cfg["n_heads"], cfg["n_kv_heads"], M, max_seq, layer_dicts, T=1,
+                            select_mode=mode, xl_depth=cfg["xl_depth"], xl_mode=xl_mode)
+
+    def time_model(m):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(st):
+            m.h.copy_(h0_dev)
+            m.decode_step(pos, stream=st)
+            st.synchronize()
+            with torch.cuda.graph(g, stream=st):
+                m.h.copy_(h0_dev, non_blocking=True)
+                m.decode_step(pos, stream=st)
+            for _ in range(3):
+                g.replay()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(st)
+            for _ in range(steps):
+                g.replay()
+            e1.record(st)
+        e1.synchronize()
+        counts = m.stats.cpu().numpy()[:, :, 0].astype(np.float64)
+        return e0.elapsed_time(e1) / steps, counts
+
+    out = {}
+    # ---- thresholds: for each (layer, operator input) the midpoint between the k-th and the
+    # (k+1)-th largest |x| of a calibration token run in top-k mode, averaged over 4 tokens ----
+    cal = model(layers, afx.MODE_TOPK, afx.XL_OFF)
+    tau = np.zeros((NL, 4))
+    n_cal = 4
+    bufs = ((afx.BUF_XNORM, afx.OP_QKV), (afx.BUF_ATTN, 0), (afx.BUF_XNORM, afx.OP_GU), (afx.BUF_HM, 0))
+    tdt = torch.bfloat16 if cfg["dtype"] == "bf16" else torch.float16
+    for c in range(n_cal):
+        hc = torch.from_numpy(synth.hidden_state(cfg["seed"], 700 + c, 1, H, scale=1.0, scales_stream=6)).cuda()
+        cal.h.copy_(hc)
+        for l in range(NL):
+            cal.layer_step(l, pos)
+            for op, (which, sub) in enumerate(bufs):
+                mag = cal.bits(which, sub).view(tdt).float().abs().flatten()
+                top = torch.topk(mag, k[op] + 1).values
+                tau[l, op] += float(top[k[op] - 1] + top[k[op]]) / 2 / n_cal
+    cal.close()
+    th_layers = [dict(L, tau=[float(t) for t in tau[l]]) for l, L in enumerate(layers)]
+    m = model(th_layers, afx.MODE_THRESHOLD, afx.XL_BOOKKEEP)
+    ms, counts = time_model(m)
+    kept = counts.sum(0) / (NL * np.array(K_op, np.float64))
+    n_qkv = (cfg["n_heads"] + 2 * cfg["n_kv_heads"]) * 128
+    w_bytes = 2.0 * (counts[:, 0].sum() * n_qkv + counts[:, 1].sum() * H + counts[:, 2].sum() * 2 * M + counts[:, 3].sum() * H)
+    out["threshold_mode"] = {"tokens_per_s": round(1e3 / ms, 2), "ms_per_step": round(ms, 4),
+                             "kept_fraction": dict(zip(["qkv", "o", "gate_up", "down"], kept.round(4).tolist())),
+                             "active_weight_gbs": round(w_bytes / (ms * 1e-3) / 1e9, 1),
+                             "calibration": f"{n_cal} other tokens, target keep {100 - cfg['sparsity_percent']}%"}
+    m.close()
+    m = model(layers, afx.MODE_TOPK, afx.XL_REUSE)
+    ms, counts = time_model(m)
+    out["cross_layer_reuse_mode"] = {"tokens_per_s": round(1e3 / ms, 2), "ms_per_step": round(ms, 4),
+                                     "note": "layers 3g+1..3g+3 compute on layer 3g's active sets (top-k 50%)"}
+    m.close()
+    return out
+
+
 def active_bytes_per_token(cfg, k):
     H, M = cfg["hidden"], cfg["mlp"]
     n_qkv = (cfg["n_heads"] + 2 * cfg["n_kv_heads"]) * 128
@@ -260,6 +334,8 @@ def run_afx(args):
     pred = stats[1:]
     precision = (pred[:, :, 1].sum(0) / np.maximum(pred[:, :, 0].sum(0), 1)).round(4).tolist()
 
+    variants = run_variants(cfg, layers, k, h0_dev, pos, st, min(args.steps, 50)) if not args.no_variants else None
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu = cpu_baseline(cfg, layers, k, h0_host.numpy(), pos)
@@ -282,6 +358,7 @@ def run_afx(args):
             "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline, "cpu_baseline": cpu, "clocks": clocks,
             "cross_layer_precision": dict(zip(["qkv", "o", "gate_up", "down"], precision)),
+            "variants": variants,
         }
         print(json.dumps(line))
     if world > 1:
@@ -373,6 +450,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="afx", choices=["afx", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-variants", action="store_true", help="skip the threshold / reuse variants")
     ap.add_argument("--layers", type=int, default=0, help="run only the first N layers (profiling aid)")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -20,7 +20,7 @@ constexpr int kAttnWarps = kAttnThreads / 32;
 constexpr int kAttnWorkers = 2 * kAttnWarps;  // half warps: each walks its own positions
 constexpr int kHeadDim = 128;
 constexpr int kAttnMaxRep = 8;  // query heads per kv head
-constexpr int kAttnUnroll = 4;  // cache rows (K and V each) in flight per half warp
+constexpr int kAttnUnroll = 4;  // cache rows (K and V each) in flight per half warp (8 with one query head)
 
 struct AttnArgs {
     const float* qkv;  // [T][n_qkv] fp32: q heads | k heads | v heads
@@ -125,7 +125,7 @@ __device__ __forceinline__ void attention_block(const AttnArgs& a, AttnSmem* sm)
         for (int j = 0; j < 8; ++j) acc[r][j] = 0.0f;
     }
 
-    constexpr int U = kAttnUnroll;
+    constexpr int U = REP == 1 ? 2 * kAttnUnroll : kAttnUnroll;
     for (int p0 = l_lo + worker; p0 < l_hi; p0 += kAttnWorkers * U) {
         uint4 kraw[U], vraw[U];
 #pragma unroll
