@@ -33,7 +33,7 @@ CFG = dict(name="llama7b_decode_32L_bf16_top50_xl3", dtype="bf16", n_layers=32, 
 ORACLE_SAMPLE_LAYERS = 16
 # dram__bytes_read.sum + dram__bytes_write.sum of one fused gate/up launch of this workload,
 # from the ncu capture summarised in profiles/fused_op_kernel_7b_ncu_full.md (None when stale).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 94_080_256
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 95_432_448
 
 
 def measured_peaks():
@@ -345,10 +345,10 @@ def run_afx(args):
             "metric": "decode tokens/s (batch 1)", "value": round(tok_s, 2), "unit": "tokens/s",
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": round(ms / args.steps, 4), "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16 weights, fp32 accumulate", "data": "synthetic",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": cfg["name"], "layers": cfg["n_layers"], "hidden": cfg["hidden"],
                        "mlp": cfg["mlp"], "kv_past": cfg["past"], "sparsity_percent": cfg["sparsity_percent"],
-                       "select": "top-k", "cross_layer_depth": cfg["xl_depth"], "cross_layer_mode": "bookkeeping",
+                       "select": "top-k", "accumulate": "fp32", "cross_layer_depth": cfg["xl_depth"], "cross_layer_mode": "bookkeeping",
                        "l2": "6.5 GB of weights streamed per step, far larger than L2",
                        "parallelism": f"{world} independent replica(s)"},
             "active_weight_gbs": round(w_bytes / (ms / args.steps * 1e-3) / 1e9, 1),
