@@ -227,14 +227,28 @@ __device__ __forceinline__ void attention_block(const AttnArgs& a, AttnSmem* sm)
     cluster.sync();
     for (int e = rank + S * tid; e < rep * kHeadDim; e += S * kAttnThreads) {
         const int r = e / kHeadDim, d = e - r * kHeadDim;
+        // all remote reads first (they are independent), then the merge in block order
+        float mq[8], aq[8], lq[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            mq[q] = -INFINITY;
+            aq[q] = 0.0f;
+            lq[q] = 0.0f;
+            if (q < S) {
+                mq[q] = cluster.map_shared_rank(&sm->part_m[0], q)[r];
+                aq[q] = cluster.map_shared_rank(&sm->part_acc[0][0], q)[r * kHeadDim + d];
+                lq[q] = cluster.map_shared_rank(&sm->part_l[0], q)[r];
+            }
+        }
         float M = -INFINITY;
-        for (int q = 0; q < S; ++q) M = fmaxf(M, cluster.map_shared_rank(&sm->part_m[0], q)[r]);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) M = fmaxf(M, mq[q]);
         float num = 0.0f, den = 0.0f;
-        for (int q = 0; q < S; ++q) {
-            const float mq = cluster.map_shared_rank(&sm->part_m[0], q)[r];
-            const float w = mq == -INFINITY ? 0.0f : fast_exp2(mq - M);
-            num = fmaf(w, cluster.map_shared_rank(&sm->part_acc[0][0], q)[r * kHeadDim + d], num);
-            den = fmaf(w, cluster.map_shared_rank(&sm->part_l[0], q)[r], den);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const float w = mq[q] == -INFINITY ? 0.0f : fast_exp2(mq[q] - M);
+            num = fmaf(w, aq[q], num);
+            den = fmaf(w, lq[q], den);
         }
         a.out[static_cast<size_t>(t) * a.q_heads * kHeadDim + static_cast<size_t>(hk * rep + r) * kHeadDim + d] =
             float_to_bits<DT>(num / den);
