@@ -77,7 +77,7 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
     const bool topk = own && a.mode == AFX_MODE_TOPK && a.k > 0 && a.k < K;
     AFX_MARK(0);
     cluster_arrive();
-    if (topk) block_clear_key_hist(hist);  // does not depend on the previous kernel
+    if (topk) block_clear_key_hist<kGemvThreads>(hist);  // does not depend on the previous kernel
 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");

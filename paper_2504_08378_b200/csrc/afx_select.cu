@@ -28,7 +28,7 @@ select_kernel(const uint16_t* __restrict__ x, int K, int T, int mode, int k, flo
         uint16_t* xs = reinterpret_cast<uint16_t*>(s_dyn + flag_bytes);
         uint32_t* hist = reinterpret_cast<uint32_t*>(s_dyn + flag_bytes + (static_cast<size_t>(K) + 7) / 8 * 8 * 2);
         const bool topk = mode == AFX_MODE_TOPK && k > 0 && k < K;
-        if (topk) block_clear_key_hist(hist);
+        if (topk) block_clear_key_hist<kSelectThreads>(hist);
         unsigned long long fl = 0ull;
         int pos0 = 0, total = 0;
         for (int t = 0; t < T; ++t) {

@@ -92,10 +92,29 @@ __device__ __forceinline__ void chunk_keys(const uint16_t* xs, int c, uint32_t (
     }
 }
 
+// Two 15-bit keys per 32-bit word (bits 15 and 31 clear), compared at once against a key
+// replicated in both halves: the result has bit 15 / bit 31 set where the low / high key
+// satisfies the relation.  (0x8000 | key) - (thr + 1) stays within its 16 bits -- no borrow
+// crosses the halves -- and keeps bit 15 exactly when key > thr; likewise for equality.
+constexpr uint32_t kHalfTops = 0x80008000u;
+__device__ __forceinline__ uint32_t swar_pair(uint32_t key) { return key * 0x00010001u; }
+__device__ __forceinline__ uint32_t swar_gt(uint32_t keys2, uint32_t thr2_plus1) {
+    return ((keys2 | kHalfTops) - thr2_plus1) & kHalfTops;
+}
+__device__ __forceinline__ uint32_t swar_eq(uint32_t keys2, uint32_t thr2) {
+    return ~(((keys2 ^ thr2) | kHalfTops) - 0x00010001u) & kHalfTops;
+}
+// The two mask bits of word i of a chunk as bits 2i and 2i+1 of the chunk's flag byte.
+__device__ __forceinline__ uint32_t swar_byte_bits(uint32_t mask, int i) {
+    return (((mask >> 15) & 1u) | ((mask >> 30) & 2u)) << (2 * i);
+}
+
 // Sets the key histogram to zero (no barrier).
+template <int NT>
 __device__ __forceinline__ void block_clear_key_hist(uint32_t* hist) {
-    for (int i = threadIdx.x; i < kKeyHistWords / 4; i += blockDim.x)
-        reinterpret_cast<uint4*>(hist)[i] = make_uint4(0u, 0u, 0u, 0u);
+    uint4* h4 = reinterpret_cast<uint4*>(hist) + threadIdx.x;
+#pragma unroll
+    for (int i = 0; i < kKeyHistWords / 4 / NT; ++i) h4[i * NT] = make_uint4(0u, 0u, 0u, 0u);
 }
 
 // The k-th largest magnitude key (1 <= k <= K) of xs[0..K) (shared memory, 16-byte aligned,
@@ -115,25 +134,27 @@ __device__ __forceinline__ void block_kth_key(const uint16_t* xs, int K, int k, 
     int c_lo, c_hi;
     thread_chunk_range(K, c_lo, c_hi);
     for (int c = c_lo; c < c_hi; ++c) {
-        uint32_t key[8];
-        chunk_keys(xs, c, key);
+        const uint4 raw = *reinterpret_cast<const uint4*>(xs + (c << 3));
+        const uint32_t r[4] = {raw.x, raw.y, raw.z, raw.w};
+        const int nvalid = K - (c << 3);  // < 8 only in the last chunk of a K that is no multiple of 8
 #pragma unroll
-        for (int e = 0; e < 8; ++e)
-            if ((c << 3) + e < K) atomicAdd(&hist[key[e] >> 1], 1u << ((key[e] & 1u) << 4));
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t k0 = r[i] & 0x7FFFu, k1 = (r[i] >> 16) & 0x7FFFu;
+            if (2 * i < nvalid) atomicAdd(&hist[k0 >> 1], (k0 & 1u) ? 0x10000u : 1u);
+            if (2 * i + 1 < nvalid) atomicAdd(&hist[k1 >> 1], (k1 & 1u) ? 0x10000u : 1u);
+        }
     }
     __syncthreads();
     // counters of this warp's slice, highest keys last: row i, lane l holds words
     // warp*W + (i*32 + l)*4 .. +4
     const uint32_t* mine = hist + warp * W + lane * 4;
-    int rowsum[NR];
-    int lane_total = 0;
+    uint32_t packed = 0;  // two 16-bit sums, neither overflows (K <= 32768)
 #pragma unroll
     for (int i = 0; i < NR; ++i) {
         const uint4 v = *reinterpret_cast<const uint4*>(mine + i * 128);
-        const uint32_t p = v.x + v.y + v.z + v.w;  // two 16-bit lanes, neither overflows (K <= 32768)
-        rowsum[i] = static_cast<int>((p & 0xFFFFu) + (p >> 16));
-        lane_total += rowsum[i];
+        packed += v.x + v.y + v.z + v.w;
     }
+    const int lane_total = static_cast<int>((packed & 0xFFFFu) + (packed >> 16));
     const int warp_total = __reduce_add_sync(0xFFFFFFFFu, lane_total);
     int total;
     const int below = warp_prefix(warp_total, s->wtot[0], total);
@@ -142,6 +163,13 @@ __device__ __forceinline__ void block_kth_key(const uint16_t* xs, int K, int k, 
         int rem = k - above;                       // rank from the top inside this warp's slice
         int row = 0, row_lane_sum = 0;
         bool found = false;
+        int rowsum[NR];
+#pragma unroll
+        for (int i = 0; i < NR; ++i) {
+            const uint4 v = *reinterpret_cast<const uint4*>(mine + i * 128);
+            const uint32_t p = v.x + v.y + v.z + v.w;
+            rowsum[i] = static_cast<int>((p & 0xFFFFu) + (p >> 16));
+        }
 #pragma unroll
         for (int i = NR - 1; i >= 0; --i) {
             const int rt = __reduce_add_sync(0xFFFFFFFFu, rowsum[i]);
@@ -241,23 +269,32 @@ __device__ __forceinline__ unsigned long long block_token_flags(const uint16_t* 
         return fl;
     }
     if (!hist_clean) {
-        block_clear_key_hist(hist);
+        block_clear_key_hist<NT>(hist);
         __syncthreads();
     }
     uint32_t thr;
     int need_eq, tot_eq;
     block_kth_key<NT>(xs, K, k, hist, s, thr, need_eq, tot_eq);
-    // channels above the k-th key are in; of those equal to it, the need_eq lowest ids
+    // Channels above the k-th key are in; of those equal to it, the need_eq lowest ids.
+    // Full chunks are handled two keys per operation (swar_*); a partial last chunk is padded
+    // with zeros in shared memory, and a zero key can only count as "equal" when thr == 0, so
+    // its padding is masked out of the equality masks.
+    const uint32_t thr2 = swar_pair(thr), thr2p1 = swar_pair(thr + 1u);
     int g = 0, e_cnt = 0;
     for (int c = c_lo; c < c_hi; ++c) {
-        uint32_t key[8];
-        chunk_keys(xs, c, key);
+        const uint4 raw = *reinterpret_cast<const uint4*>(xs + (c << 3));
+        const uint32_t r[4] = {raw.x & 0x7FFF7FFFu, raw.y & 0x7FFF7FFFu, raw.z & 0x7FFF7FFFu, raw.w & 0x7FFF7FFFu};
+        const int nvalid = K - (c << 3);
+        uint32_t gm = 0, em = 0;  // the four words' masks shifted apart: popc counts all eight keys
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const bool in = (c << 3) + e < K;
-            g += in && key[e] > thr;
-            e_cnt += in && key[e] == thr;
+        for (int i = 0; i < 4; ++i) {
+            uint32_t e = swar_eq(r[i], thr2);
+            if (nvalid < 8) e &= (2 * i < nvalid ? 0x8000u : 0u) | (2 * i + 1 < nvalid ? 0x80000000u : 0u);
+            gm |= swar_gt(r[i], thr2p1) >> i;
+            em |= e >> i;
         }
+        g += __popc(gm);
+        e_cnt += __popc(em);
     }
     int pre_e = 0;
     if (single) {
@@ -270,24 +307,41 @@ __device__ __forceinline__ unsigned long long block_token_flags(const uint16_t* 
         int tot;
         pre_e = block_prefix(e_cnt, s->wtot[1], tot);
     }
+    const bool all_eq = need_eq == tot_eq;
     int seen_e = pre_e;
     int pos = pos0;
     for (int c = c_lo; c < c_hi; ++c) {
         const uint4 raw = *reinterpret_cast<const uint4*>(xs + (c << 3));
-        const uint32_t r[4] = {raw.x, raw.y, raw.z, raw.w};
-        uint32_t byte = 0;
+        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+        const int nvalid = K - (c << 3);
+        uint32_t byte = 0, eq_byte = 0;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const uint32_t bits = (r[e >> 1] >> (16 * (e & 1))) & 0xFFFFu;
-            const uint32_t key = bits & 0x7FFFu;
-            const bool in = (c << 3) + e < K;
-            const bool eq = in && key == thr;
-            const bool pred = in && (key > thr || (eq && (need_eq == tot_eq || seen_e < need_eq)));
-            seen_e += eq;
-            byte |= static_cast<uint32_t>(pred) << e;
-            if (single && pred) emit((c << 3) + e, pos++, static_cast<uint16_t>(bits));
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t keys2 = w[i] & 0x7FFF7FFFu;
+            uint32_t e = swar_eq(keys2, thr2);
+            if (nvalid < 8) e &= (2 * i < nvalid ? 0x8000u : 0u) | (2 * i + 1 < nvalid ? 0x80000000u : 0u);
+            byte |= swar_byte_bits(swar_gt(keys2, thr2p1), i);
+            eq_byte |= swar_byte_bits(e, i);
+        }
+        if (all_eq) {
+            byte |= eq_byte;
+        } else {
+            // ties across the boundary: the equal channels are kept in channel order until
+            // need_eq of them (over the whole vector) are in
+            while (eq_byte != 0u) {
+                const uint32_t low = eq_byte & (0u - eq_byte);
+                eq_byte ^= low;
+                if (seen_e < need_eq) byte |= low;
+                ++seen_e;
+            }
         }
         fl |= static_cast<unsigned long long>(byte) << (8 * (c - c_lo));
+        if (single) {
+            for (uint32_t rest = byte; rest != 0u; rest &= rest - 1u) {
+                const int e = __ffs(static_cast<int>(rest)) - 1;
+                emit((c << 3) + e, pos++, xs[(c << 3) + e]);
+            }
+        }
     }
     return fl;
 }
