@@ -80,13 +80,22 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
     if (topk) block_clear_key_hist<kGemvThreads>(hist);  // does not depend on the previous kernel
 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // the norm's gains are weights: they can be on their way before the wait for h
+    constexpr int NH = 4;  // float4 pieces of h (and of the gain) a thread keeps in registers
+    float4 gv[NH];
+    if (IN == IN_NORM) {
+#pragma unroll
+        for (int i = 0; i < NH; ++i) {
+            const int c = tid + i * kGemvThreads;
+            gv[i] = c < (K >> 2) ? reinterpret_cast<const float4*>(a.gain)[c] : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        }
+    }
     asm volatile("griddepcontrol.wait;" ::: "memory");
     AFX_MARK(1);
 
     // ---- input stage --------------------------------------------------------------------
     if (IN == IN_NORM) {
         // x = round(h / rms(h) * gain), every block for itself (K % 8 == 0, 16-byte aligned rows)
-        constexpr int NH = 4;  // float4 pieces of h a thread keeps between the two passes
         const int nq = K >> 2;
         for (int t = 0; t < T; ++t) {
             const float4* ht = reinterpret_cast<const float4*>(a.h + static_cast<size_t>(t) * K);
@@ -117,8 +126,7 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
             for (int w = 0; w < kGemvWarps; ++w) tot += red16[w];
             const float inv = 1.0f / sqrtf(tot / static_cast<float>(K) + a.eps);
             const float4* gq = reinterpret_cast<const float4*>(a.gain);
-            auto emit = [&](int c, const float4& v) {
-                const float4 g = gq[c];
+            auto emit = [&](int c, const float4& v, const float4& g) {
                 const uint32_t lo = static_cast<uint32_t>(float_to_bits<DT>(v.x * inv * g.x)) |
                                     (static_cast<uint32_t>(float_to_bits<DT>(v.y * inv * g.y)) << 16);
                 const uint32_t hi = static_cast<uint32_t>(float_to_bits<DT>(v.z * inv * g.z)) |
@@ -130,9 +138,9 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
 #pragma unroll
             for (int i = 0; i < NH; ++i) {
                 const int c = tid + i * kGemvThreads;
-                if (c < nq) emit(c, hv[i]);
+                if (c < nq) emit(c, hv[i], gv[i]);
             }
-            for (int c = tid + NH * kGemvThreads; c < nq; c += kGemvThreads) emit(c, ht[c]);
+            for (int c = tid + NH * kGemvThreads; c < nq; c += kGemvThreads) emit(c, ht[c], gq[c]);
         }
         __syncthreads();
     }
@@ -170,7 +178,7 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
                             sm->col[p] = j;
                             sm->xv[0][p] = bits_to_float<DT>(bits);
                         }
-                    });
+                    }, e_lo, e_lo + e_n);
                 first_staged = true;
             } else {
                 fl |= block_token_flags<DT, kGemvThreads>(xt, K, a.mode, a.k, a.tau, hist, t == 0, sel, T == 1,

@@ -229,7 +229,8 @@ __device__ __forceinline__ void block_kth_key(const uint16_t* xs, int K, int k, 
 // already zero and visible.  With `single` set (the token is the only one) the call also
 // returns the list position of the thread's first active channel in `pos0` and the length
 // of the list in `cnt`, from the same scan that orders the tie-break, and calls
-// emit(channel, list position, 16-bit pattern) for every active channel of the thread.
+// emit(channel, list position, 16-bit pattern) for the thread's active channels (in top-k
+// mode only for a thread that can own a position in [emit_lo, emit_hi)).
 struct NoEmit {
     __device__ __forceinline__ void operator()(int, int, uint16_t) const {}
 };
@@ -238,7 +239,8 @@ template <int DT, int NT, class Emit = NoEmit>
 __device__ __forceinline__ unsigned long long block_token_flags(const uint16_t* xs, int K, int mode, int k,
                                                                 float tau, uint32_t* hist, bool hist_clean,
                                                                 SelectScratch* s, bool single, int& pos0,
-                                                                int& cnt, Emit emit = Emit()) {
+                                                                int& cnt, Emit emit = Emit(), int emit_lo = 0,
+                                                                int emit_hi = 0x7FFFFFFF) {
     int c_lo, c_hi;
     thread_chunk_range(K, c_lo, c_hi);
     unsigned long long fl = 0ull;
@@ -308,6 +310,7 @@ __device__ __forceinline__ unsigned long long block_token_flags(const uint16_t* 
         pre_e = block_prefix(e_cnt, s->wtot[1], tot);
     }
     const bool all_eq = need_eq == tot_eq;
+    const bool emits = single && pos0 < emit_hi && pos0 + g + e_cnt > emit_lo;
     int seen_e = pre_e;
     int pos = pos0;
     for (int c = c_lo; c < c_hi; ++c) {
@@ -336,7 +339,7 @@ __device__ __forceinline__ unsigned long long block_token_flags(const uint16_t* 
             }
         }
         fl |= static_cast<unsigned long long>(byte) << (8 * (c - c_lo));
-        if (single) {
+        if (emits) {
             for (uint32_t rest = byte; rest != 0u; rest &= rest - 1u) {
                 const int e = __ffs(static_cast<int>(rest)) - 1;
                 emit((c << 3) + e, pos++, xs[(c << 3) + e]);
