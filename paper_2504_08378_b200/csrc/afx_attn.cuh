@@ -81,13 +81,31 @@ __device__ __forceinline__ void attention_block(const AttnArgs& a, AttnSmem* sm)
     const uint32_t half_mask = 0xFFFFu << (16 * half);  // the two halves of a warp work on different keys
 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    uint16_t* kc = a.k_cache + static_cast<size_t>(t) * a.max_seq * a.kv_heads * kHeadDim;
+    uint16_t* vc = a.v_cache + static_cast<size_t>(t) * a.max_seq * a.kv_heads * kHeadDim;
+    // With one query head per kv head the registers allow it: the past rows of this half
+    // warp's first batch do not depend on the kernel that is still running (they were written
+    // by earlier tokens), so they are requested before the wait for q, k, v.
+    constexpr int U = REP == 1 ? 2 * kAttnUnroll : kAttnUnroll;
+    constexpr bool kEarly = REP == 1;
+    uint4 kraw[U], vraw[U];
+    if (kEarly) {
+        const size_t rs = static_cast<size_t>(a.kv_heads) * kHeadDim;
+        const size_t ho = static_cast<size_t>(hk) * kHeadDim + l16 * 8;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int p = l_lo + worker + u * kAttnWorkers;
+            if (p < l_hi && p < a.pos) {
+                kraw[u] = *reinterpret_cast<const uint4*>(kc + static_cast<size_t>(p) * rs + ho);
+                vraw[u] = *reinterpret_cast<const uint4*>(vc + static_cast<size_t>(p) * rs + ho);
+            }
+        }
+    }
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
     const float* row = a.qkv + static_cast<size_t>(t) * a.n_qkv;
     const float* cs = a.rope_cos + static_cast<size_t>(a.pos) * (kHeadDim / 2);
     const float* sn = a.rope_sin + static_cast<size_t>(a.pos) * (kHeadDim / 2);
-    uint16_t* kc = a.k_cache + static_cast<size_t>(t) * a.max_seq * a.kv_heads * kHeadDim;
-    uint16_t* vc = a.v_cache + static_cast<size_t>(t) * a.max_seq * a.kv_heads * kHeadDim;
     const size_t row_stride = static_cast<size_t>(a.kv_heads) * kHeadDim;
     const size_t head_off = static_cast<size_t>(hk) * kHeadDim + l16 * 8;
 
@@ -125,17 +143,20 @@ __device__ __forceinline__ void attention_block(const AttnArgs& a, AttnSmem* sm)
         for (int j = 0; j < 8; ++j) acc[r][j] = 0.0f;
     }
 
-    constexpr int U = REP == 1 ? 2 * kAttnUnroll : kAttnUnroll;
-    for (int p0 = l_lo + worker; p0 < l_hi; p0 += kAttnWorkers * U) {
-        uint4 kraw[U], vraw[U];
+    // rows of a batch that are not in registers yet: all of them, or (first batch, requested
+    // before the wait) only the row this kernel has just appended
+    auto fetch = [&](int p0, bool only_new) {
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int p = p0 + u * kAttnWorkers;
-            if (p < l_hi) {
+            if (p < l_hi && (!only_new || p >= a.pos)) {
                 kraw[u] = *reinterpret_cast<const uint4*>(kc + static_cast<size_t>(p) * row_stride + head_off);
                 vraw[u] = *reinterpret_cast<const uint4*>(vc + static_cast<size_t>(p) * row_stride + head_off);
             }
         }
+    };
+    fetch(l_lo + worker, kEarly);
+    for (int p0 = l_lo + worker; p0 < l_hi; p0 += kAttnWorkers * U) {
         float sc[REP][U];
 #pragma unroll
         for (int r = 0; r < REP; ++r) {
@@ -189,6 +210,7 @@ __device__ __forceinline__ void attention_block(const AttnArgs& a, AttnSmem* sm)
                 }
             }
         }
+        if (p0 + kAttnWorkers * U < l_hi) fetch(p0 + kAttnWorkers * U, false);
     }
 
     // meet the half warps of the block (fixed order), one query head at a time
