@@ -443,6 +443,102 @@ def run_reference(args):
     }))
 
 
+def run_cache70b(args):
+    """Workload 5: a 70B-shaped stack whose weights live in pinned host memory (standing in for
+    flash) behind a hot-channel cache in HBM sized to 30 % of each operator.  Per decode step
+    and operator: selection (top 50 %), afx_cache_fetch (LFU policy + copy of the misses over
+    PCIe), sparse GEMV through the slot list.  The operator inputs are synthesised per (step,
+    layer, operator) with Zipf(1.1)-skewed channel activity, not chained.  Prints one JSON line:
+    cache hit rate, host->HBM bytes per token, tokens/s."""
+    import numpy as np
+    import torch
+    from paper_2504_08378_b200 import afx, synth
+    torch.cuda.set_device(0)
+    dt, hidden, mlp, n_q, n_kv = "bf16", 8192, 28672, 64, 8
+    n_layers, steps = (args.layers or 8), args.cache_steps
+    ops = [("qkv", hidden, (n_q + 2 * n_kv) * 128), ("o", n_q * 128, hidden), ("gate_up", hidden, 2 * mlp),
+           ("down", mlp, hidden)]
+    st = torch.cuda.Stream()
+    caches = []
+    host_bytes = 0
+    for l in range(n_layers):
+        for oi, (name, K, N) in enumerate(ops):
+            w_dev = synth.device_normal_bits(5, 1000 * (l + 1) + oi, (K, N), 0.02, dt)
+            w_host = torch.empty((K, N), dtype=torch.int16).pin_memory()
+            w_host.copy_(w_dev)
+            del w_dev
+            k = synth.keep_count(K, 50)
+            C = (K * 30) // 100
+            slots = torch.empty((C + k, N), dtype=torch.int16, device="cuda")
+            handle = afx.afx_cache_create(afx.CacheDesc(dtype=afx.DTYPES[dt], K=K, N=N, ldw=N, capacity=C,
+                                                        staging_rows=k, host_base=w_host.data_ptr(),
+                                                        slots=slots.data_ptr()))
+            caches.append(dict(name=name, K=K, N=N, k=k, host=w_host, slots=slots, handle=handle,
+                               stats=torch.zeros(3, dtype=torch.int64, device="cuda"),
+                               stream_id=100 * l + oi))
+            host_bytes += K * N * 2
+    Kmax, Nmax = max(o[1] for o in ops), max(o[2] for o in ops)
+    idx = torch.empty(Kmax, dtype=torch.int32, device="cuda")
+    cnt = torch.zeros(1, dtype=torch.int32, device="cuda")
+    slot_out = torch.empty(Kmax, dtype=torch.int32, device="cuda")
+    y = torch.empty((1, Nmax), dtype=torch.float32, device="cuda")
+    tdt = torch.bfloat16
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(55)
+    # channel popularity: weight r^-1.1 over a seeded permutation per operator, shared by all steps
+    for c in caches:
+        perm = torch.randperm(c["K"], generator=gen, device="cuda")
+        rank = torch.empty(c["K"], device="cuda")
+        rank[perm] = torch.arange(1, c["K"] + 1, device="cuda", dtype=torch.float32)
+        c["logw"] = -1.1 * torch.log(rank)
+    hits = {o[0]: 0 for o in ops}
+    misses = {o[0]: 0 for o in ops}
+    fetched_bytes = 0
+    active_bytes = 0
+    ms_total = 0.0
+    overflow = 0
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(st):
+        for step in range(steps):
+            xs = []
+            for c in caches:  # this step's operator inputs (input generation, not timed)
+                u = torch.rand(c["K"], generator=gen, device="cuda").clamp_(1e-7, 1 - 1e-7)
+                score = c["logw"] - torch.log(-torch.log(u))
+                sign = torch.where(torch.rand(c["K"], generator=gen, device="cuda") < 0.5, -1.0, 1.0)
+                xs.append((torch.exp(score / 4.0) * sign).to(tdt).view(torch.int16))
+            ev0.record(st)
+            for c, x in zip(caches, xs):
+                afx.afx_select_active(x, dt, c["K"], 1, afx.MODE_TOPK, c["k"], 0.0, idx, cnt, None, stream=st)
+                afx.afx_cache_fetch(c["handle"], idx, cnt, slot_out, c["stats"], stream=st)
+                afx.afx_sparse_gemv(c["slots"], dt, c["K"], c["N"], c["N"], x, 1, idx, cnt, slot_out, y, 0, stream=st)
+            ev1.record(st)
+            ev1.synchronize()
+            ms_total += ev0.elapsed_time(ev1)
+            for c in caches:
+                sv = afx.CacheStats.from_buffer_copy(c["stats"].cpu().numpy().tobytes())
+                hits[c["name"]] += sv.hits
+                misses[c["name"]] += sv.misses
+                fetched_bytes += sv.bytes_fetched
+                overflow += sv.overflow
+                active_bytes += c["k"] * c["N"] * 2
+    for c in caches:
+        afx.afx_cache_destroy(c["handle"])
+    th, tm = sum(hits.values()), sum(misses.values())
+    print(json.dumps({
+        "metric": "cache hit rate and host->HBM bytes per token (weights in pinned host memory, 30% HBM cache)",
+        "value": round(th / max(th + tm, 1), 4), "unit": "hit rate", "n_gpus": 1, "steps": steps, "warmup": 0,
+        "ms_per_step": round(ms_total / steps, 3), "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "llama70b_shaped_%dL_hostweights_cache30_zipf1.1_top50" % n_layers, "hidden": hidden,
+                   "mlp": mlp, "q_heads": n_q, "kv_heads": n_kv, "host_weight_bytes": host_bytes,
+                   "cache_fraction": 0.3, "cold_start": True},
+        "hit_rate_per_operator": {n: round(hits[n] / max(hits[n] + misses[n], 1), 4) for n in hits},
+        "host_to_hbm_bytes_per_token": int(fetched_bytes / steps),
+        "host_to_hbm_fraction_of_active_bytes": round(fetched_bytes / max(active_bytes, 1), 4),
+        "tokens_per_s": round(steps / (ms_total * 1e-3), 2), "pcie_gbs": round(fetched_bytes / (ms_total * 1e-3) / 1e9, 1),
+        "staging_overflow": int(overflow),
+        "paper_context": "the paper reports 74-77% context-level hit rate and an 18% load share with a 50% cache (Sec. 7.3)"}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -452,9 +548,14 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-variants", action="store_true", help="skip the threshold / reuse variants")
     ap.add_argument("--layers", type=int, default=0, help="run only the first N layers (profiling aid)")
+    ap.add_argument("--workload", default="decode7b", choices=["decode7b", "cache70b"],
+                    help="decode7b: the headline decode token; cache70b: host-resident weights behind the LFU cache")
+    ap.add_argument("--cache-steps", type=int, default=256, help="decode steps of the cache70b workload")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "cache70b":
+        run_cache70b(args)
     else:
         run_afx(args)
 
