@@ -201,7 +201,11 @@ afx_status afx_state_destroy(afx_state* state);
 #define AFX_BUF_IDX 5        /* int32 [K_op]          active list last used by operator input `op` */
 #define AFX_BUF_MISS 6       /* int32 [K_op]          A \ P of the last bookkeeping            */
 #define AFX_BUF_STATS 7      /* int32 [n_layers][4][4] per layer and op: list length, |A & P|,  */
-                             /*                       |A \ P|, 0 (written by each layer step)  */
+                             /*                       |A \ P| (written by each layer step), and */
+                             /*                       0x10000 | the k-th largest magnitude key  */
+                             /*                       of the last one-token top-k selection (0  */
+                             /*                       before the first; the next token's search */
+                             /*                       starts there, any value gives the same set) */
 afx_status afx_state_buffer(const afx_state* state, int which, int op, void** ptr, size_t* bytes);
 
 /*

@@ -36,6 +36,9 @@ struct FusedArgs {
     int32_t* miss_out;            // ... A \ P ascending (capacity K)
     int32_t* miss_count;
     int32_t* hit_count;           // |A & P|
+    // ---- top-k search hint (may be NULL): 0x10000 | k-th key of this operator's last top-k
+    // selection with T == 1; read before the selection, rewritten after it by block (0,0) ----
+    int32_t* kth_slot;
 };
 
 // Dynamic shared memory: [16-bit inputs: T tokens (IN_NORM) or one token (IN_X), each padded
@@ -89,6 +92,14 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
             const int c = tid + i * kGemvThreads;
             gv[i] = c < (K >> 2) ? reinterpret_cast<const float4*>(a.gain)[c] : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
         }
+    }
+    // the hint was written by an earlier token's launch of this operator, not by the kernel
+    // waited for below (a launch that reads the value its own scribe block has just rewritten
+    // only gets a better hint: the selection's result does not depend on it)
+    uint32_t hint = kNoKeyHint;
+    if (topk && T == 1 && a.kth_slot != nullptr) {
+        const uint32_t v = static_cast<uint32_t>(__ldcg(a.kth_slot));
+        if (v & 0x10000u) hint = v & 0x7FFFu;
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");
     AFX_MARK(1);
@@ -178,8 +189,9 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
                             sm->col[p] = j;
                             sm->xv[0][p] = bits_to_float<DT>(bits);
                         }
-                    }, e_lo, e_lo + e_n);
+                    }, e_lo, e_lo + e_n, hint);
                 first_staged = true;
+                if (scribe && tid == 0 && a.kth_slot != nullptr) *a.kth_slot = 0x10000 | sel->res[0];
             } else {
                 fl |= block_token_flags<DT, kGemvThreads>(xt, K, a.mode, a.k, a.tau, hist, t == 0, sel, T == 1,
                                                           pos0, cnt);

@@ -293,6 +293,7 @@ static void plan_selection(const afx_model* m, const afx_state* s, int layer, in
     a->miss_out = nullptr;
     a->miss_count = nullptr;
     a->hit_count = nullptr;
+    a->kth_slot = my_stats + 3;
     const int depth = d.xl_depth;
     if (!cross_layer || depth <= 0 || d.xl_mode == AFX_XL_OFF) return;
     const bool predictor = (layer % depth) == 0;

@@ -17,6 +17,8 @@
 // the same arguments.
 #pragma once
 
+#include <type_traits>
+
 #include "afx_common.cuh"
 
 namespace afx {
@@ -94,19 +96,12 @@ __device__ __forceinline__ void chunk_keys(const uint16_t* xs, int c, uint32_t (
 
 // Two 15-bit keys per 32-bit word (bits 15 and 31 clear), compared at once against a key
 // replicated in both halves: the result has bit 15 / bit 31 set where the low / high key
-// satisfies the relation.  (0x8000 | key) - (thr + 1) stays within its 16 bits -- no borrow
-// crosses the halves -- and keeps bit 15 exactly when key > thr; likewise for equality.
+// is greater.  (0x8000 | key) - (thr + 1) stays within its 16 bits -- no borrow crosses the
+// halves -- and keeps bit 15 exactly when key > thr.
 constexpr uint32_t kHalfTops = 0x80008000u;
 __device__ __forceinline__ uint32_t swar_pair(uint32_t key) { return key * 0x00010001u; }
 __device__ __forceinline__ uint32_t swar_gt(uint32_t keys2, uint32_t thr2_plus1) {
     return ((keys2 | kHalfTops) - thr2_plus1) & kHalfTops;
-}
-__device__ __forceinline__ uint32_t swar_eq(uint32_t keys2, uint32_t thr2) {
-    return ~(((keys2 ^ thr2) | kHalfTops) - 0x00010001u) & kHalfTops;
-}
-// The two mask bits of word i of a chunk as bits 2i and 2i+1 of the chunk's flag byte.
-__device__ __forceinline__ uint32_t swar_byte_bits(uint32_t mask, int i) {
-    return (((mask >> 15) & 1u) | ((mask >> 30) & 2u)) << (2 * i);
 }
 
 // Sets the key histogram to zero (no barrier).
@@ -223,24 +218,153 @@ __device__ __forceinline__ void block_kth_key(const uint16_t* xs, int K, int k, 
     tot_eq = s->res[2];
 }
 
+// Keys searched around a hint of the k-th key: about +-19 % in magnitude for either type.
+template <int DT>
+struct KeyWindow {
+    static constexpr int kBins = DT == AFX_BF16 ? 64 : 512;
+};
+constexpr uint32_t kNoKeyHint = 0xFFFFFFFFu;
+
+// block_kth_key with a hint (a key near the expected answer, e.g. the one found for the
+// previous token): counts the keys above a window of KeyWindow<DT>::kBins keys around the hint
+// and histograms only the keys inside it -- two masked compares per word and a few
+// uncontended atomics instead of one atomic per key, and one warp resolves the window.
+// Exact whenever it returns true; returns false (same value in every thread, outputs
+// untouched, `hist` clean again) when the k-th key lies outside the window.  `hist` as for
+// block_kth_key; words [0, kBins] are left dirty.
+template <int DT, int NT>
+__device__ __forceinline__ bool block_kth_key_near(const uint16_t* xs, int K, int k, uint32_t hint,
+                                                   uint32_t* hist, SelectScratch* s, uint32_t& thr,
+                                                   int& need_eq, int& tot_eq) {
+    constexpr int WB = KeyWindow<DT>::kBins;
+    constexpr int P = WB / 32;  // bins per lane of the resolving warp
+    static_assert(P == 2 || P % 4 == 0, "window bins per lane: 2 or a multiple of 4");
+    const int lane = lane_id();
+    const int lo = max(0, min(static_cast<int>(hint & 0x7FFFu) - WB / 2, 32768 - WB));
+    // swar_gt(keys, pair(v)) marks keys >= v (it tests key > v - 1); lo + WB <= 0x8000 keeps
+    // the subtraction inside its half
+    const uint32_t lo2 = swar_pair(static_cast<uint32_t>(lo)), hi2 = swar_pair(static_cast<uint32_t>(lo + WB));
+    int c_lo, c_hi;
+    thread_chunk_range(K, c_lo, c_hi);
+    int above = 0;
+    for (int c = c_lo; c < c_hi; ++c) {
+        const uint4 raw = *reinterpret_cast<const uint4*>(xs + (c << 3));
+        const uint32_t r[4] = {raw.x & 0x7FFF7FFFu, raw.y & 0x7FFF7FFFu, raw.z & 0x7FFF7FFFu, raw.w & 0x7FFF7FFFu};
+        const int nvalid = K - (c << 3);
+        uint32_t am = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t a = swar_gt(r[i], hi2);
+            uint32_t in = swar_gt(r[i], lo2) & ~a;
+            // the zero padding of a partial last chunk would fall into a window that starts at 0
+            if (nvalid < 8) in &= (2 * i < nvalid ? 0x8000u : 0u) | (2 * i + 1 < nvalid ? 0x80000000u : 0u);
+            am |= a >> i;
+            if (in & 0x8000u) atomicAdd(&hist[(r[i] & 0xFFFFu) - lo], 1u);
+            if (in & 0x80000000u) atomicAdd(&hist[(r[i] >> 16) - lo], 1u);
+        }
+        above += __popc(am);
+    }
+    above = __reduce_add_sync(0xFFFFFFFFu, above);
+    if (lane == 0 && above != 0) atomicAdd(&hist[WB], static_cast<uint32_t>(above));
+    __syncthreads();
+    if (warp_id() == 0) {
+        const int ab = static_cast<int>(hist[WB]);
+        uint32_t cnt[P];
+        if (P == 2) {
+            const uint2 v = *reinterpret_cast<const uint2*>(hist + lane * 2);
+            cnt[0] = v.x;
+            cnt[1] = v.y;
+        } else {
+#pragma unroll
+            for (int q = 0; q < P / 4; ++q) {
+                const uint4 v = *reinterpret_cast<const uint4*>(hist + lane * P + q * 4);
+                cnt[4 * q] = v.x;
+                cnt[4 * q + 1] = v.y;
+                cnt[4 * q + 2] = v.z;
+                cnt[4 * q + 3] = v.w;
+            }
+        }
+        int lane_sum = 0;
+#pragma unroll
+        for (int q = 0; q < P; ++q) lane_sum += static_cast<int>(cnt[q]);
+        int suf = lane_sum;  // inclusive suffix sums: higher lanes hold higher keys
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int n = __shfl_down_sync(0xFFFFFFFFu, suf, o);
+            if (lane + o < 32) suf += n;
+        }
+        const int inside = __shfl_sync(0xFFFFFFFFu, suf, 0);
+        const bool ok = ab < k && k <= ab + inside;
+        if (ok) {
+            int rem = k - ab;  // rank from the top inside the window
+            const uint32_t has = __ballot_sync(0xFFFFFFFFu, suf >= rem);
+            if (lane == 31 - __clz(static_cast<int>(has))) {
+                rem -= suf - lane_sum;
+                bool done = false;
+#pragma unroll
+                for (int q = P - 1; q >= 0; --q) {
+                    const int cq = static_cast<int>(cnt[q]);
+                    if (!done) {
+                        if (rem <= cq) {
+                            done = true;
+                            s->res[0] = lo + lane * P + q;
+                            s->res[1] = rem;
+                            s->res[2] = cq;
+                        } else {
+                            rem -= cq;
+                        }
+                    }
+                }
+            }
+        }
+        if (lane == 0) s->res[3] = ok ? 1 : 0;
+    }
+    __syncthreads();
+    if (s->res[3] == 0) {
+        for (int i = threadIdx.x; i <= WB; i += NT) hist[i] = 0u;
+        __syncthreads();
+        return false;
+    }
+    thr = static_cast<uint32_t>(s->res[0]);
+    need_eq = s->res[1];
+    tot_eq = s->res[2];
+    return true;
+}
+
 // Active flags of ONE token for the calling thread's chunks: byte v of the result covers the
 // 8 channels of chunk c_lo + v (bit e = channel 8 * (c_lo + v) + e).  xs as for
 // block_kth_key.  `hist` is the key histogram (top-k only); `hist_clean` says that it is
 // already zero and visible.  With `single` set (the token is the only one) the call also
 // returns the list position of the thread's first active channel in `pos0` and the length
 // of the list in `cnt`, from the same scan that orders the tie-break, and calls
-// emit(channel, list position, 16-bit pattern) for the thread's active channels (in top-k
-// mode only for a thread that can own a position in [emit_lo, emit_hi)).
+// emit(channel, list position, 16-bit pattern) for the thread's active channels (only for a
+// thread that can own a position in [emit_lo, emit_hi)).  `hint` (top-k,
+// `single` only; kNoKeyHint = none) is a guess of the k-th key that shortens the search and
+// never changes the result.  After a top-k selection with 0 < k < K, s->res[0] holds the k-th
+// key until the next selection.
 struct NoEmit {
     __device__ __forceinline__ void operator()(int, int, uint16_t) const {}
 };
+
+// emit(channel, list position, 16-bit pattern) for the set bits of chunk c's flag byte (w = the
+// chunk's four words); the first set bit gets position `pos`.  Eight independent predicated
+// calls, no loop over the set bits: nothing waits for the previous channel.
+template <class Emit>
+__device__ __forceinline__ void emit_chunk(uint32_t byte, int c, const uint32_t (&w)[4], int pos, Emit& emit) {
+#pragma unroll
+    for (int e = 0; e < 8; ++e)
+        if (byte & (1u << e))
+            emit((c << 3) + e, pos + __popc(byte & ((1u << e) - 1u)),
+                 static_cast<uint16_t>(w[e >> 1] >> (16 * (e & 1))));
+}
 
 template <int DT, int NT, class Emit = NoEmit>
 __device__ __forceinline__ unsigned long long block_token_flags(const uint16_t* xs, int K, int mode, int k,
                                                                 float tau, uint32_t* hist, bool hist_clean,
                                                                 SelectScratch* s, bool single, int& pos0,
                                                                 int& cnt, Emit emit = Emit(), int emit_lo = 0,
-                                                                int emit_hi = 0x7FFFFFFF) {
+                                                                int emit_hi = 0x7FFFFFFF,
+                                                                uint32_t hint = kNoKeyHint) {
     int c_lo, c_hi;
     thread_chunk_range(K, c_lo, c_hi);
     unsigned long long fl = 0ull;
@@ -263,9 +387,15 @@ __device__ __forceinline__ unsigned long long block_token_flags(const uint16_t* 
         if (single) {
             pos0 = block_prefix(__popcll(fl), s->wtot[1], cnt);
             int pos = pos0;
-            for (unsigned long long rest = fl; rest != 0ull; rest &= rest - 1ull) {
-                const int j = (c_lo << 3) + __ffsll(static_cast<long long>(rest)) - 1;
-                emit(j, pos++, xs[j]);
+            if (!std::is_same<Emit, NoEmit>::value && pos0 < emit_hi && pos0 + __popcll(fl) > emit_lo) {
+                for (int c = c_lo; c < c_hi; ++c) {
+                    const uint32_t byte = static_cast<uint32_t>(fl >> (8 * (c - c_lo))) & 0xFFu;
+                    if (byte == 0u) continue;
+                    const uint4 raw = *reinterpret_cast<const uint4*>(xs + (c << 3));
+                    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+                    emit_chunk(byte, c, w, pos, emit);
+                    pos += __popc(byte);
+                }
             }
         }
         return fl;
@@ -276,28 +406,32 @@ __device__ __forceinline__ unsigned long long block_token_flags(const uint16_t* 
     }
     uint32_t thr;
     int need_eq, tot_eq;
-    block_kth_key<NT>(xs, K, k, hist, s, thr, need_eq, tot_eq);
-    // Channels above the k-th key are in; of those equal to it, the need_eq lowest ids.
-    // Full chunks are handled two keys per operation (swar_*); a partial last chunk is padded
-    // with zeros in shared memory, and a zero key can only count as "equal" when thr == 0, so
-    // its padding is masked out of the equality masks.
+    if (!(single && hint != kNoKeyHint && block_kth_key_near<DT, NT>(xs, K, k, hint, hist, s, thr, need_eq, tot_eq)))
+        block_kth_key<NT>(xs, K, k, hist, s, thr, need_eq, tot_eq);
+    // Channels above the k-th key are in; of those equal to it, the need_eq lowest ids.  One
+    // pass over the thread's chunks, two keys per operation (swar_*), leaves two flag sets in
+    // registers: keys greater than the k-th and keys equal to it.  A partial last chunk is
+    // padded with zeros in shared memory; a zero key is never greater, and counts as equal
+    // only when thr == 0, so the padding is masked out of the equal flags.
     const uint32_t thr2 = swar_pair(thr), thr2p1 = swar_pair(thr + 1u);
-    int g = 0, e_cnt = 0;
+    unsigned long long fg = 0ull, fe = 0ull;
     for (int c = c_lo; c < c_hi; ++c) {
         const uint4 raw = *reinterpret_cast<const uint4*>(xs + (c << 3));
         const uint32_t r[4] = {raw.x & 0x7FFF7FFFu, raw.y & 0x7FFF7FFFu, raw.z & 0x7FFF7FFFu, raw.w & 0x7FFF7FFFu};
-        const int nvalid = K - (c << 3);
-        uint32_t gm = 0, em = 0;  // the four words' masks shifted apart: popc counts all eight keys
+        uint32_t gt = 0, ge = 0;  // word i: low key -> bit 2i, high key -> bit 16 + 2i
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            uint32_t e = swar_eq(r[i], thr2);
-            if (nvalid < 8) e &= (2 * i < nvalid ? 0x8000u : 0u) | (2 * i + 1 < nvalid ? 0x80000000u : 0u);
-            gm |= swar_gt(r[i], thr2p1) >> i;
-            em |= e >> i;
+            gt |= (swar_gt(r[i], thr2p1) >> (15 - 2 * i)) & (0x00010001u << (2 * i));
+            ge |= (swar_gt(r[i], thr2) >> (15 - 2 * i)) & (0x00010001u << (2 * i));  // key > thr - 1
         }
-        g += __popc(gm);
-        e_cnt += __popc(em);
+        const uint32_t gbyte = (gt | (gt >> 15)) & 0xFFu;
+        uint32_t ebyte = (ge | (ge >> 15)) & 0xFFu & ~gbyte;
+        const int nvalid = K - (c << 3);
+        if (nvalid < 8) ebyte &= (1u << nvalid) - 1u;
+        fg |= static_cast<unsigned long long>(gbyte) << (8 * (c - c_lo));
+        fe |= static_cast<unsigned long long>(ebyte) << (8 * (c - c_lo));
     }
+    const int g = __popcll(fg), e_cnt = __popcll(fe);
     int pre_e = 0;
     if (single) {
         int tot;
@@ -309,40 +443,30 @@ __device__ __forceinline__ unsigned long long block_token_flags(const uint16_t* 
         int tot;
         pre_e = block_prefix(e_cnt, s->wtot[1], tot);
     }
-    const bool all_eq = need_eq == tot_eq;
-    const bool emits = single && pos0 < emit_hi && pos0 + g + e_cnt > emit_lo;
-    int seen_e = pre_e;
-    int pos = pos0;
-    for (int c = c_lo; c < c_hi; ++c) {
-        const uint4 raw = *reinterpret_cast<const uint4*>(xs + (c << 3));
-        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-        const int nvalid = K - (c << 3);
-        uint32_t byte = 0, eq_byte = 0;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const uint32_t keys2 = w[i] & 0x7FFF7FFFu;
-            uint32_t e = swar_eq(keys2, thr2);
-            if (nvalid < 8) e &= (2 * i < nvalid ? 0x8000u : 0u) | (2 * i + 1 < nvalid ? 0x80000000u : 0u);
-            byte |= swar_byte_bits(swar_gt(keys2, thr2p1), i);
-            eq_byte |= swar_byte_bits(e, i);
+    fl = fg;
+    if (need_eq == tot_eq) {
+        fl |= fe;
+    } else {
+        // ties across the boundary: the equal channels are kept in channel order until
+        // need_eq of them (over the whole vector) are in
+        int seen_e = pre_e;
+        for (unsigned long long rest = fe; rest != 0ull && seen_e < need_eq; ++seen_e) {
+            const unsigned long long low = rest & (0ull - rest);
+            rest ^= low;
+            fl |= low;
         }
-        if (all_eq) {
-            byte |= eq_byte;
-        } else {
-            // ties across the boundary: the equal channels are kept in channel order until
-            // need_eq of them (over the whole vector) are in
-            while (eq_byte != 0u) {
-                const uint32_t low = eq_byte & (0u - eq_byte);
-                eq_byte ^= low;
-                if (seen_e < need_eq) byte |= low;
-                ++seen_e;
-            }
-        }
-        fl |= static_cast<unsigned long long>(byte) << (8 * (c - c_lo));
-        if (emits) {
-            for (uint32_t rest = byte; rest != 0u; rest &= rest - 1u) {
-                const int e = __ffs(static_cast<int>(rest)) - 1;
-                emit((c << 3) + e, pos++, xs[(c << 3) + e]);
+    }
+    if (single && !std::is_same<Emit, NoEmit>::value) {
+        const int n = __popcll(fl);
+        if (pos0 < emit_hi && pos0 + n > emit_lo) {
+            int pos = pos0;
+            for (int c = c_lo; c < c_hi; ++c) {
+                const uint32_t byte = static_cast<uint32_t>(fl >> (8 * (c - c_lo))) & 0xFFu;
+                if (byte == 0u) continue;
+                const uint4 raw = *reinterpret_cast<const uint4*>(xs + (c << 3));
+                const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+                emit_chunk(byte, c, w, pos, emit);
+                pos += __popc(byte);
             }
         }
     }
@@ -367,10 +491,12 @@ __device__ __forceinline__ void for_each_owned_active(unsigned long long fl, int
     int c_lo, c_hi;
     thread_chunk_range(K, c_lo, c_hi);
     int pos = pos0;
-    while (fl != 0ull) {
-        const int b = __ffsll(static_cast<long long>(fl)) - 1;
-        fl &= fl - 1ull;
-        f((c_lo << 3) + b, pos++);
+    for (int c = c_lo; c < c_hi; ++c) {
+        const uint32_t byte = static_cast<uint32_t>(fl >> (8 * (c - c_lo))) & 0xFFu;
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+            if (byte & (1u << e)) f((c << 3) + e, pos + __popc(byte & ((1u << e) - 1u)));
+        pos += __popc(byte);
     }
 }
 

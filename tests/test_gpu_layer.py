@@ -175,3 +175,55 @@ def test_mlp_block_threshold_sweep(dt):
         y_ref = oracle.sparse_gemv(L["w_down"], dt, hidden, hm_gpu, idx_d)
         assert rel_err(y.cpu().numpy(), y_ref) <= TOL
         m.close()
+
+
+def kth_key(bits, k):
+    keys = np.sort(bits.reshape(-1).astype(np.int64) & 0x7FFF)
+    return int(keys[keys.size - k])
+
+
+@pytest.mark.parametrize("ties", [False, True])
+@pytest.mark.parametrize("dt", ["bf16", "f16"])
+def test_topk_search_hint_never_changes_the_selection(dt, ties):
+    """Each one-token top-k selection records its k-th key; the next token's search starts in
+    a window around it.  Whatever that hint is -- exact, a few keys off, at the window's
+    edges, far outside, the extremes, absent -- every stage still matches the oracle, with
+    many equal magnitudes at the boundary too."""
+    heads, kvh, T, max_seq, pos = 4, 4, 1, 48, 37
+    hidden, mlp = heads * 128, 1384
+    cfg = ol.Config(dt, hidden, heads, kvh, mlp, mode=oracle.TOPK)
+    L = synth.layer_weights(33, 0, hidden, heads, kvh, mlp, dt, gain_jitter=0.0 if ties else 0.1)
+    k = [synth.keep_count(K, 50) for K in (hidden, heads * 128, hidden, mlp)]
+    L["k"] = k
+    kc0, vc0 = synth.kv_cache(33, 0, T, max_seq, kvh, pos)
+    L["k_cache"], L["v_cache"] = kc0, vc0
+    h0 = synth.hidden_state(33, 5, T, hidden)
+    if ties:
+        h0 = np.round(h0 * 1.5).astype(np.float32)  # a handful of distinct magnitudes
+    lw = oracle_weights(L, k)
+    m = make(cfg, [L], T, afx.MODE_TOPK, max_seq=max_seq)
+    half = 32 if dt == "bf16" else 256
+
+    def run(hints):
+        m.h.copy_(torch.from_numpy(h0).cuda())
+        if hints is not None:
+            m.stats[0, :, 3] = torch.tensor(hints, dtype=torch.int32, device="cuda")
+        m.layer_step(0, pos)
+        torch.cuda.synchronize()
+        out = check_layer_stages(cfg, L, lw, m, 0, h0, kc0, vc0, pos, T)
+        assert [len(i) for i in out["idx"]] == k
+        return out
+
+    run(None)  # state just created: no hint
+    inputs = [bits_np(m.bits(afx.BUF_XNORM, afx.OP_QKV)), bits_np(m.bits(afx.BUF_ATTN)),
+              bits_np(m.bits(afx.BUF_XNORM, afx.OP_GU)), bits_np(m.bits(afx.BUF_HM))]
+    exact = [kth_key(b, kk) for b, kk in zip(inputs, k)]
+    assert m.stats.cpu().numpy()[0, :, 3].tolist() == [0x10000 | e for e in exact]
+    clamp = lambda v: min(0x7FFF, max(0, v))
+    for delta in (0, 1, -1, 7, half - 1, -half, half, -half - 1, 5 * half, -5 * half):
+        out = run([0x10000 | clamp(e + delta) for e in exact])
+        assert out["stats"][:, 3].tolist() == [0x10000 | e for e in exact], delta
+    for raw in (0x10000, 0x10000 | 0x7FFF, 0, 0x7FFF, -1):
+        out = run([raw] * 4)
+        assert out["stats"][:, 3].tolist() == [0x10000 | e for e in exact], raw
+    m.close()
