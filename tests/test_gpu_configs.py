@@ -57,7 +57,7 @@ def test_config2_mlp_block_7b_threshold_sweep():
         m.close()
 
 
-def _run_layers(cfg, layers_dev, layers_host, k, T, pos, max_seq, seed, xl_depth=0, xl_mode=0):
+def _run_layers(cfg, layers_dev, layers_host, k, T, pos, max_seq, seed, xl_depth=0, xl_mode=0, warm_tokens=0):
     kvh = cfg.n_kv_heads
     caches = []
     for l, dev in enumerate(layers_dev):
@@ -65,6 +65,12 @@ def _run_layers(cfg, layers_dev, layers_host, k, T, pos, max_seq, seed, xl_depth
         dev["k_cache"], dev["v_cache"] = kc0, vc0
         caches.append((kc0, vc0))
     m = make(cfg, layers_dev, T, afx.MODE_TOPK, xl_depth=xl_depth, xl_mode=xl_mode, max_seq=max_seq)
+    for w in range(warm_tokens):  # earlier, different tokens: they leave their k-th keys as search hints
+        m.h.copy_(torch.from_numpy(synth.hidden_state(seed, 105 + w, T, cfg.hidden, scales_stream=6)).cuda())
+        for l in range(len(layers_host)):
+            m.layer_step(l, pos)
+        torch.cuda.synchronize()
+        assert (m.stats.cpu().numpy()[:, :, 3] >> 16 == 1).all()
     h = synth.hidden_state(seed, 5, T, cfg.hidden, scales_stream=6)
     m.h.copy_(torch.from_numpy(h).cuda())
     prev_idx = None
@@ -93,6 +99,17 @@ def test_config3_7b_decode_layers_with_cross_layer_bookkeeping():
     pairs = [full_layer(3, l, hidden, heads, heads, mlp, dt, k=k) for l in range(2)]
     _run_layers(cfg, [p[0] for p in pairs], [p[1] for p in pairs], k, 1, 2048, 2056, 3, xl_depth=3,
                 xl_mode=afx.XL_BOOKKEEP)
+
+
+@pytest.mark.parametrize("dt", ["bf16", "f16"])
+def test_config3_7b_layer_after_other_tokens(dt):
+    """The token checked is the third one decoded: its top-k searches start from the previous
+    token's k-th keys (three 8-channel chunks per thread on the 11008-wide input)."""
+    hidden, heads, mlp = 4096, 32, 11008
+    cfg = ol.Config(dt, hidden, heads, heads, mlp, mode=oracle.TOPK)
+    k = [synth.keep_count(K, 50) for K in (hidden, heads * 128, hidden, mlp)]
+    dev, host = full_layer(6, 0, hidden, heads, heads, mlp, dt, k=k)
+    _run_layers(cfg, [dev], [host], k, 1, 2048, 2056, 6, warm_tokens=2)
 
 
 @pytest.mark.parametrize("T", [1, 4])
