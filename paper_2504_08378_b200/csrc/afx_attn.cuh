@@ -80,6 +80,7 @@ __device__ __forceinline__ void attention_block(const AttnArgs& a, AttnSmem* sm)
     const float qscale = rsqrtf(static_cast<float>(kHeadDim)) * 1.4426950408889634f;
     const uint32_t half_mask = 0xFFFFu << (16 * half);  // the two halves of a warp work on different keys
 
+    AFX_MARK(0);
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     uint16_t* kc = a.k_cache + static_cast<size_t>(t) * a.max_seq * a.kv_heads * kHeadDim;
     uint16_t* vc = a.v_cache + static_cast<size_t>(t) * a.max_seq * a.kv_heads * kHeadDim;
@@ -102,6 +103,7 @@ __device__ __forceinline__ void attention_block(const AttnArgs& a, AttnSmem* sm)
         }
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    AFX_MARK(1);
 
     const float* row = a.qkv + static_cast<size_t>(t) * a.n_qkv;
     const float* cs = a.rope_cos + static_cast<size_t>(a.pos) * (kHeadDim / 2);
@@ -155,6 +157,7 @@ __device__ __forceinline__ void attention_block(const AttnArgs& a, AttnSmem* sm)
             }
         }
     };
+    AFX_MARK(2);
     fetch(l_lo + worker, kEarly);
     for (int p0 = l_lo + worker; p0 < l_hi; p0 += kAttnWorkers * U) {
         float sc[REP][U];
@@ -213,6 +216,7 @@ __device__ __forceinline__ void attention_block(const AttnArgs& a, AttnSmem* sm)
         if (p0 + kAttnWorkers * U < l_hi) fetch(p0 + kAttnWorkers * U, false);
     }
 
+    AFX_MARK(3);
     // meet the half warps of the block (fixed order), one query head at a time
 #pragma unroll
     for (int r = 0; r < REP; ++r) {
@@ -246,7 +250,9 @@ __device__ __forceinline__ void attention_block(const AttnArgs& a, AttnSmem* sm)
             __syncthreads();
         }
     }
+    AFX_MARK(4);
     cluster.sync();
+    AFX_MARK(5);
     for (int e = rank + S * tid; e < rep * kHeadDim; e += S * kAttnThreads) {
         const int r = e / kHeadDim, d = e - r * kHeadDim;
         // all remote reads first (they are independent), then the merge in block order
@@ -275,7 +281,9 @@ __device__ __forceinline__ void attention_block(const AttnArgs& a, AttnSmem* sm)
         a.out[static_cast<size_t>(t) * a.q_heads * kHeadDim + static_cast<size_t>(hk * rep + r) * kHeadDim + d] =
             float_to_bits<DT>(num / den);
     }
+    AFX_MARK(6);
     cluster.sync();
+    AFX_MARK(7);
 }
 
 }  // namespace afx
