@@ -70,7 +70,6 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
 
     const int Kp = (K + 7) & ~7;
     uint16_t* xs = reinterpret_cast<uint16_t*>(dyn);
-    uint32_t* flags = reinterpret_cast<uint32_t*>(dyn + fused_input_smem(IN, K, T));
     unsigned char* work = dyn + fused_input_smem(IN, K, T) + fused_flag_smem(K);
     uint32_t* hist = reinterpret_cast<uint32_t*>(work);
     GemvSmem<TMAX, CAP>* sm = reinterpret_cast<GemvSmem<TMAX, CAP>*>(work);
@@ -100,6 +99,15 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
     if (topk && T == 1 && a.kth_slot != nullptr) {
         const uint32_t v = static_cast<uint32_t>(__ldcg(a.kth_slot));
         if (v & 0x10000u) hint = v & 0x7FFFu;
+    }
+    // likewise the predicted set this selection is compared with: the predictor layer wrote it
+    // several kernels ago (byte v = the flags of the v-th chunk this thread owns, like `fl`)
+    unsigned long long pm = 0ull;
+    if (scribe && own && a.bitmap_pred != nullptr) {
+        int q_lo, q_hi;
+        thread_chunk_range(K, q_lo, q_hi);
+        const uint8_t* pred = reinterpret_cast<const uint8_t*>(a.bitmap_pred);
+        for (int c = q_lo; c < q_hi; ++c) pm |= static_cast<unsigned long long>(__ldcg(pred + c)) << (8 * (c - q_lo));
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");
     AFX_MARK(1);
@@ -198,11 +206,38 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
             }
         }
         if (T > 1) pos0 = block_prefix(__popcll(fl), sel->wtot[2], cnt);
-        if (scribe) store_flag_bytes(fl, K, flags);
     } else {
         if (IN == IN_X && T == 1) block_stage_token(a.x, K, xs);
         cnt = *a.count_in;
         cnt = max(0, min(cnt, K));
+    }
+    // ---- side outputs (one block of the grid): plain stores that drain while the block streams ----
+    if (scribe) {
+        if (own) {
+            if (a.idx_out != nullptr) for_each_owned_active(fl, K, pos0, [&](int j, int pos) { a.idx_out[pos] = j; });
+            int q_lo, q_hi;
+            thread_chunk_range(K, q_lo, q_hi);
+            if (a.bitmap_out != nullptr) {  // byte c of the bitmap = the flags of chunk c
+                uint8_t* bytes = reinterpret_cast<uint8_t*>(a.bitmap_out);
+                for (int c = q_lo; c < q_hi; ++c) bytes[c] = static_cast<uint8_t>(fl >> (8 * (c - q_lo)));
+                for (int c = ((K + 7) >> 3) + tid; c < nwords * 4; c += kGemvThreads) bytes[c] = 0;
+            }
+            if (a.bitmap_pred != nullptr) {
+                // A \ P in ascending order, |A & P|
+                const unsigned long long ms = fl & ~pm;
+                int n_miss;
+                const int m0 = block_prefix(__popcll(ms), sel->wtot[3], n_miss);
+                if (a.miss_out != nullptr)
+                    for_each_owned_active(ms, K, m0, [&](int j, int pos) { a.miss_out[pos] = j; });
+                if (tid == 0) {
+                    if (a.miss_count != nullptr) *a.miss_count = n_miss;
+                    if (a.hit_count != nullptr) *a.hit_count = cnt - n_miss;
+                }
+            }
+        } else if (a.idx_out != nullptr && a.idx_out != a.idx_in) {
+            for (int i = tid; i < cnt; i += kGemvThreads) a.idx_out[i] = a.idx_in[i];
+        }
+        if (tid == 0 && a.count_out != nullptr) *a.count_out = cnt;
     }
     AFX_MARK(3);
     const int c_lo = s * cnt / S;  // S <= 8, cnt <= 2^20: no overflow
@@ -248,35 +283,6 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
     }
     AFX_MARK(5);
 
-    // ---- side outputs (one block of the grid) ---------------------------------------------
-    if (scribe) {
-        if (own) {
-            if (a.idx_out != nullptr) for_each_owned_active(fl, K, pos0, [&](int j, int pos) { a.idx_out[pos] = j; });
-            __syncthreads();  // flag bytes of every thread are in place
-            if (a.bitmap_out != nullptr)
-                for (int w = tid; w < nwords; w += kGemvThreads) a.bitmap_out[w] = flags[w];
-            if (a.bitmap_pred != nullptr) {
-                // A \ P in ascending order, |A & P|: the predicted set, byte by byte like fl
-                int q_lo, q_hi;
-                thread_chunk_range(K, q_lo, q_hi);
-                const uint8_t* pred = reinterpret_cast<const uint8_t*>(a.bitmap_pred);
-                unsigned long long pm = 0ull;
-                for (int c = q_lo; c < q_hi; ++c) pm |= static_cast<unsigned long long>(pred[c]) << (8 * (c - q_lo));
-                const unsigned long long ms = fl & ~pm;
-                int n_miss;
-                const int m0 = block_prefix(__popcll(ms), sel->wtot[3], n_miss);
-                if (a.miss_out != nullptr)
-                    for_each_owned_active(ms, K, m0, [&](int j, int pos) { a.miss_out[pos] = j; });
-                if (tid == 0) {
-                    if (a.miss_count != nullptr) *a.miss_count = n_miss;
-                    if (a.hit_count != nullptr) *a.hit_count = cnt - n_miss;
-                }
-            }
-        } else if (a.idx_out != nullptr && a.idx_out != a.idx_in) {
-            for (int i = tid; i < cnt; i += kGemvThreads) a.idx_out[i] = a.idx_in[i];
-        }
-        if (tid == 0 && a.count_out != nullptr) *a.count_out = cnt;
-    }
     AFX_MARK(6);
 
     gemv_finish_tile<DT, TMAX, PW, CAP, EP>(acc, T, tile, sm, recv, a.ep);
