@@ -180,6 +180,11 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
     // [c_lo, c_hi) of the list is known before the selection and the pass that decides the
     // flags (it has the channel's bits in registers) stages the first CAP entries directly.
     const bool early = topk && T == 1;
+    // one word per chunk, in the work area behind the staging and reduction buffers
+    constexpr size_t kXchgOffset = kKeyHistBytes - (kSelectFastMaxK / 8) * 4;
+    constexpr bool kXchgFits = sizeof(GemvSmem<TMAX, CAP>) <= kXchgOffset;
+    static_assert(TMAX > 1 || kXchgFits, "work area too small for the chunk exchange");
+    uint32_t* xchg = kXchgFits ? reinterpret_cast<uint32_t*>(work + kXchgOffset) : nullptr;
     bool first_staged = false;
     if (own) {
         const int e_lo = s * a.k / S, e_n = min(CAP, (s + 1) * a.k / S - e_lo);
@@ -197,7 +202,7 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
                             sm->col[p] = j;
                             sm->xv[0][p] = bits_to_float<DT>(bits);
                         }
-                    }, e_lo, e_lo + e_n, hint);
+                    }, e_lo, e_lo + e_n, hint, xchg);
                 first_staged = true;
                 if (scribe && tid == 0 && a.kth_slot != nullptr) *a.kth_slot = 0x10000 | sel->res[0];
             } else {

@@ -340,7 +340,9 @@ __device__ __forceinline__ bool block_kth_key_near(const uint16_t* xs, int K, in
 // emit(channel, list position, 16-bit pattern) for the thread's active channels (only for a
 // thread that can own a position in [emit_lo, emit_hi)).  `hint` (top-k,
 // `single` only; kNoKeyHint = none) is a guess of the k-th key that shortens the search and
-// never changes the result.  After a top-k selection with 0 < k < K, s->res[0] holds the k-th
+// never changes the result.  `xchg` (top-k emits; may be NULL) is ceil(K/8) words of shared
+// memory apart from the histogram's first KeyWindow bins and from whatever emit writes.
+// After a top-k selection with 0 < k < K, s->res[0] holds the k-th
 // key until the next selection.
 struct NoEmit {
     __device__ __forceinline__ void operator()(int, int, uint16_t) const {}
@@ -364,7 +366,8 @@ __device__ __forceinline__ unsigned long long block_token_flags(const uint16_t* 
                                                                 SelectScratch* s, bool single, int& pos0,
                                                                 int& cnt, Emit emit = Emit(), int emit_lo = 0,
                                                                 int emit_hi = 0x7FFFFFFF,
-                                                                uint32_t hint = kNoKeyHint) {
+                                                                uint32_t hint = kNoKeyHint,
+                                                                uint32_t* xchg = nullptr) {
     int c_lo, c_hi;
     thread_chunk_range(K, c_lo, c_hi);
     unsigned long long fl = 0ull;
@@ -457,16 +460,40 @@ __device__ __forceinline__ unsigned long long block_token_flags(const uint16_t* 
         }
     }
     if (single && !std::is_same<Emit, NoEmit>::value) {
-        const int n = __popcll(fl);
-        if (pos0 < emit_hi && pos0 + n > emit_lo) {
+        const int nchunks = (K + 7) >> 3;
+        if (xchg != nullptr && nchunks > NT) {
+            // Several chunks per thread: the few owners of the positions [emit_lo, emit_hi)
+            // would emit chunk after chunk.  Every owner posts (position, flags) of its chunks
+            // instead, and the chunks that touch the range are emitted by one thread each.
             int pos = pos0;
             for (int c = c_lo; c < c_hi; ++c) {
                 const uint32_t byte = static_cast<uint32_t>(fl >> (8 * (c - c_lo))) & 0xFFu;
-                if (byte == 0u) continue;
-                const uint4 raw = *reinterpret_cast<const uint4*>(xs + (c << 3));
-                const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-                emit_chunk(byte, c, w, pos, emit);
+                xchg[c] = (static_cast<uint32_t>(pos) << 8) | byte;
                 pos += __popc(byte);
+            }
+            __syncthreads();
+            for (int c = threadIdx.x; c < nchunks; c += NT) {
+                const uint32_t v = xchg[c];
+                const uint32_t byte = v & 0xFFu;
+                const int p = static_cast<int>(v >> 8);
+                if (byte != 0u && p < emit_hi && p + __popc(byte) > emit_lo) {
+                    const uint4 raw = *reinterpret_cast<const uint4*>(xs + (c << 3));
+                    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+                    emit_chunk(byte, c, w, p, emit);
+                }
+            }
+        } else {
+            const int n = __popcll(fl);
+            if (pos0 < emit_hi && pos0 + n > emit_lo) {
+                int pos = pos0;
+                for (int c = c_lo; c < c_hi; ++c) {
+                    const uint32_t byte = static_cast<uint32_t>(fl >> (8 * (c - c_lo))) & 0xFFu;
+                    if (byte == 0u) continue;
+                    const uint4 raw = *reinterpret_cast<const uint4*>(xs + (c << 3));
+                    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+                    emit_chunk(byte, c, w, pos, emit);
+                    pos += __popc(byte);
+                }
             }
         }
     }
