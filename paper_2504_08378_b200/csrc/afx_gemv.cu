@@ -31,6 +31,7 @@ int sm_count() {
 }
 
 int g_force_pw = 0, g_force_s = 0;  // experiment knobs, 0 = automatic
+int g_cluster_margin = -1;          // experiment knob, < 0 = automatic
 
 template <int DT, int TMAX>
 static afx_status launch_gemv_t(const GemvListArgs& a, cudaStream_t st) {
@@ -60,6 +61,7 @@ extern "C" void afx_internal_tune_gemv(int pw, int s) {
     afx::g_force_pw = pw;
     afx::g_force_s = s;
 }
+extern "C" void afx_internal_cluster_margin(int margin) { afx::g_cluster_margin = margin; }
 
 extern "C" afx_status afx_sparse_gemv(const void* Wt, int dtype, int K, int N, int64_t ldw,
                                       const void* x, int T, const int32_t* idx, const int32_t* count,

@@ -86,6 +86,9 @@ struct GemvShapeChoice {
 // Widest tile and largest cluster such that all tiles' clusters are resident at once
 // (one wave) and the block count is as large as possible.  kerns[i] is the kernel
 // instantiated for tile width 256 >> i.
+extern int g_force_pw, g_force_s;  // experiment knobs (0 = automatic)
+extern int g_cluster_margin;      // experiment knob (< 0 = automatic)
+
 inline GemvShapeChoice choose_gemv_shape(int N, const void* const kerns[3], size_t dyn_smem,
                                          int force_pw = 0, int force_s = 0) {
     GemvShapeChoice best = {64, 1, (N + 63) / 64};
@@ -97,7 +100,11 @@ inline GemvShapeChoice choose_gemv_shape(int N, const void* const kerns[3], size
         int s_fit = 0;
         for (int S = kMaxCluster; S >= 1; --S) {
             if (force_s && S != force_s) continue;
-            if (max_active_clusters(kerns[i], S, dyn_smem) >= tiles) {
+            // The occupancy query counts free block slots per GPC; launched behind another
+            // kernel, two clusters fewer than it reports were seen resident at once (the
+            // last ones then ran as a second wave), so a margin stays free.
+            const int margin = g_cluster_margin >= 0 ? g_cluster_margin : (tiles + 15) / 16 < 2 ? 2 : (tiles + 15) / 16;
+            if (max_active_clusters(kerns[i], S, dyn_smem) >= tiles + margin) {
                 s_fit = S;
                 break;
             }
@@ -137,7 +144,5 @@ inline afx_status launch_clustered(Kern kern, int S, int tiles, size_t dyn_smem,
     cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, kern, a) == cudaSuccess ? AFX_OK : AFX_ERR_CUDA;
 }
-
-extern int g_force_pw, g_force_s;  // experiment knobs (0 = automatic)
 
 }  // namespace afx

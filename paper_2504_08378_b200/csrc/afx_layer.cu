@@ -549,3 +549,14 @@ extern "C" afx_status afx_mlp_block_noalloc(const void* w_gu, const void* w_down
     a.ep = {y, nullptr, hidden};
     return launch_fused<IN_X, EP_STORE>(dtype, a, st);
 }
+
+// Not part of the ABI: clusters of S blocks of the bf16 one-token operator (tile width pw,
+// plain input of K channels, h += epilogue) that the occupancy query reports as co-resident.
+extern "C" int afx_internal_max_clusters(int pw, int S, int K) {
+    using namespace afx;
+    const size_t dyn = fused_dyn_smem(IN_X, K, 1);
+    const void* kern = pw == 256 ? reinterpret_cast<const void*>(fused_op_kernel<AFX_BF16, 1, 256, IN_X, EP_ACCUM>)
+                     : pw == 128 ? reinterpret_cast<const void*>(fused_op_kernel<AFX_BF16, 1, 128, IN_X, EP_ACCUM>)
+                                 : reinterpret_cast<const void*>(fused_op_kernel<AFX_BF16, 1, 64, IN_X, EP_ACCUM>);
+    return max_active_clusters(kern, S, dyn);
+}
