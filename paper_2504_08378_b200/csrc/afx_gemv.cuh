@@ -132,6 +132,15 @@ __device__ __forceinline__ void gemv_finish_tile(float (&acc)[TMAX][8], int T, i
         }
     }
     float* dst = cluster.map_shared_rank(&recv->v[0], owner);
+    // EP_ACCUM: the value this thread will add to (first element it finishes) is asked for now,
+    // so that its latency passes behind the reduction and the cluster barrier
+    float y_old = 0.0f;
+    if (EP == EP_ACCUM && threadIdx.x < T * W) {
+        const int t = threadIdx.x / W, sl = threadIdx.x - t * W;
+        const int o = sl * S + rank;
+        const int out = tile * PW + o;
+        if (o < PW && out < ep.N) y_old = ep.y[static_cast<size_t>(t) * ep.N + out];
+    }
     if (pending_wait) cluster_wait();  // pairs with the cluster_arrive() at kernel start: all peers are running
 #pragma unroll
     for (int t = 0; t < TMAX; ++t) {
@@ -183,7 +192,7 @@ __device__ __forceinline__ void gemv_finish_tile(float (&acc)[TMAX][8], int T, i
                 float s = 0.0f;
                 for (int q = 0; q < S; ++q) s += mine[(q * T + t) * W + sl];
                 float* p = ep.y + static_cast<size_t>(t) * ep.N + out;
-                *p = (EP == EP_ACCUM) ? *p + s : s;
+                *p = (EP == EP_ACCUM) ? (e < kGemvThreads ? y_old : *p) + s : s;
             }
         }
     }
