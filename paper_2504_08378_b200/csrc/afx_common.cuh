@@ -9,15 +9,17 @@
 
 // Stage marks for kernel timing studies: compiled out unless AFX_TRACE is defined, in which
 // case thread 0 of every block stores the SM clock of mark i (0..14) into afx_trace_buf, in
-// one of four regions told apart by the launch shape (256-thread blocks; 5-, 3- and other
-// cluster widths), slots 15 and 14 of a block holding the global nanosecond timer and the SM
+// one of five regions told apart by the launch shape (256-thread blocks; 5-, 3- and other
+// cluster widths, the last split by dynamic shared memory above / below 80 KB), slots 15 and 14 of a block holding the global nanosecond timer and the SM
 // id at its mark 0.
 #ifdef AFX_TRACE
 extern __device__ long long afx_trace_buf[];
 #define AFX_MARK(i)                                                                                   \
     do {                                                                                              \
         if (threadIdx.x == 0) {                                                                       \
-            const int region_ = blockDim.x == 256 ? 0 : (gridDim.x == 5 ? 1 : (gridDim.x == 3 ? 2 : 3)); \
+            unsigned dyn_;                                                                            \
+            asm volatile("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn_));                            \
+            const int region_ = blockDim.x == 256 ? 0 : (gridDim.x == 5 ? 1 : (gridDim.x == 3 ? 2 : (dyn_ > 80000u ? 3 : 4))); \
             long long* slot_ = afx_trace_buf + (region_ * 512 + (blockIdx.y * gridDim.x + blockIdx.x) % 512) * 16; \
             slot_[(i)] = clock64();                                                                   \
             if ((i) == 0) {                                                                           \

@@ -39,6 +39,10 @@ struct FusedArgs {
     // ---- top-k search hint (may be NULL): 0x10000 | k-th key of this operator's last top-k
     // selection with T == 1; read before the selection, rewritten after it by block (0,0) ----
     int32_t* kth_slot;
+    // ---- set by the launcher: 1 if the grid has one more cluster than column tiles; its block 0
+    // repeats input stage and selection only to write the side outputs, off the path of the
+    // clusters that stream (its other blocks leave at once) ----
+    int side_cluster;
 };
 
 // Dynamic shared memory: [16-bit inputs: T tokens (IN_NORM) or one token (IN_X), each padded
@@ -65,7 +69,13 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
     const int warp = tid >> 5;
     const int S = gridDim.x, s = blockIdx.x, tile = blockIdx.y;
     const int T = a.T, K = a.K;
-    const bool scribe = (blockIdx.x == 0 && blockIdx.y == 0);  // writes the side outputs
+    const bool side = a.side_cluster != 0 && blockIdx.y == gridDim.y - 1;  // the cluster without a tile
+    if (side && blockIdx.x != 0) {
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+        return;
+    }
+    // writes the side outputs: block 0 of the side cluster, else block (0,0) next to its GEMV work
+    const bool scribe = a.side_cluster != 0 ? side : (blockIdx.x == 0 && blockIdx.y == 0);
     const int nwords = (K + 31) >> 5;
 
     const int Kp = (K + 7) & ~7;
@@ -78,7 +88,7 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
     const bool own = (a.idx_in == nullptr);
     const bool topk = own && a.mode == AFX_MODE_TOPK && a.k > 0 && a.k < K;
     AFX_MARK(0);
-    cluster_arrive();
+    if (!side) cluster_arrive();  // the side cluster never meets
     if (topk) block_clear_key_hist<kGemvThreads>(hist);  // does not depend on the previous kernel
 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -243,6 +253,7 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
             for (int i = tid; i < cnt; i += kGemvThreads) a.idx_out[i] = a.idx_in[i];
         }
         if (tid == 0 && a.count_out != nullptr) *a.count_out = cnt;
+        if (side) return;
     }
     AFX_MARK(3);
     const int c_lo = s * cnt / S;  // S <= 8, cnt <= 2^20: no overflow

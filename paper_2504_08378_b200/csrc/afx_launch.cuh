@@ -90,7 +90,7 @@ extern int g_force_pw, g_force_s;  // experiment knobs (0 = automatic)
 extern int g_cluster_margin;      // experiment knob (< 0 = automatic)
 
 inline GemvShapeChoice choose_gemv_shape(int N, const void* const kerns[3], size_t dyn_smem,
-                                         int force_pw = 0, int force_s = 0) {
+                                         int force_pw = 0, int force_s = 0, int extra_clusters = 0) {
     GemvShapeChoice best = {64, 1, (N + 63) / 64};
     int best_blocks = -1;
     for (int i = 0; i < 3; ++i) {
@@ -104,7 +104,7 @@ inline GemvShapeChoice choose_gemv_shape(int N, const void* const kerns[3], size
             // kernel, two clusters fewer than it reports were seen resident at once (the
             // last ones then ran as a second wave), so a margin stays free.
             const int margin = g_cluster_margin >= 0 ? g_cluster_margin : (tiles + 15) / 16 < 2 ? 2 : (tiles + 15) / 16;
-            if (max_active_clusters(kerns[i], S, dyn_smem) >= tiles + margin) {
+            if (max_active_clusters(kerns[i], S, dyn_smem) >= tiles + extra_clusters + margin) {
                 s_fit = S;
                 break;
             }

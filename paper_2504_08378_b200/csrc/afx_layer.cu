@@ -45,11 +45,18 @@ static afx_status launch_fused_t(const FusedArgs& a, cudaStream_t st) {
     const void* kerns[3] = {reinterpret_cast<const void*>(fused_op_kernel<DT, TMAX, 256, IN, EP>),
                             reinterpret_cast<const void*>(fused_op_kernel<DT, TMAX, 128, IN, EP>),
                             reinterpret_cast<const void*>(fused_op_kernel<DT, TMAX, 64, IN, EP>)};
-    const GemvShapeChoice c = choose_gemv_shape(a.N, kerns, dyn, g_force_pw, g_force_s);
+    // side outputs, if any, come from one more cluster than there are column tiles
+    FusedArgs b = a;
+    b.side_cluster = (a.idx_out != nullptr || a.count_out != nullptr || a.bitmap_out != nullptr ||
+                      a.xnorm_out != nullptr || a.bitmap_pred != nullptr || a.kth_slot != nullptr)
+                         ? 1 : 0;
+    const GemvShapeChoice c = choose_gemv_shape(a.N, kerns, dyn, g_force_pw, g_force_s, b.side_cluster);
+    if (c.tiles + b.side_cluster > 65535) return AFX_ERR_CAPACITY;
+    const int rows = c.tiles + b.side_cluster;
     switch (c.pw) {
-        case 256: return launch_clustered(fused_op_kernel<DT, TMAX, 256, IN, EP>, c.S, c.tiles, dyn, a, st);
-        case 128: return launch_clustered(fused_op_kernel<DT, TMAX, 128, IN, EP>, c.S, c.tiles, dyn, a, st);
-        default: return launch_clustered(fused_op_kernel<DT, TMAX, 64, IN, EP>, c.S, c.tiles, dyn, a, st);
+        case 256: return launch_clustered(fused_op_kernel<DT, TMAX, 256, IN, EP>, c.S, rows, dyn, b, st);
+        case 128: return launch_clustered(fused_op_kernel<DT, TMAX, 128, IN, EP>, c.S, rows, dyn, b, st);
+        default: return launch_clustered(fused_op_kernel<DT, TMAX, 64, IN, EP>, c.S, rows, dyn, b, st);
     }
 }
 
