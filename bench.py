@@ -33,7 +33,7 @@ CFG = dict(name="llama7b_decode_32L_bf16_top50_xl3", dtype="bf16", n_layers=32, 
 ORACLE_SAMPLE_LAYERS = 16
 # dram__bytes_read.sum + dram__bytes_write.sum of one fused gate/up launch of this workload,
 # from the ncu capture summarised in profiles/fused_op_kernel_7b_ncu_full.md (None when stale).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 94_469_888
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 94_490_368
 
 
 def measured_peaks():
