@@ -231,7 +231,8 @@ constexpr uint32_t kNoKeyHint = 0xFFFFFFFFu;
 // uncontended atomics instead of one atomic per key, and one warp resolves the window.
 // Exact whenever it returns true; returns false (same value in every thread, outputs
 // untouched, `hist` clean again) when the k-th key lies outside the window.  `hist` as for
-// block_kth_key; words [0, kBins] are left dirty.
+// block_kth_key; words [0, kBins) are left dirty and may be rewritten only after the block's
+// next barrier (the warps read them at their own pace).
 template <int DT, int NT>
 __device__ __forceinline__ bool block_kth_key_near(const uint16_t* xs, int K, int k, uint32_t hint,
                                                    uint32_t* hist, SelectScratch* s, uint32_t& thr,
@@ -264,70 +265,72 @@ __device__ __forceinline__ bool block_kth_key_near(const uint16_t* xs, int K, in
         }
         above += __popc(am);
     }
+    AFX_MARK(11);
     above = __reduce_add_sync(0xFFFFFFFFu, above);
-    if (lane == 0 && above != 0) atomicAdd(&hist[WB], static_cast<uint32_t>(above));
+    if (lane == 0) s->wtot[0][warp_id()] = above;
+    AFX_MARK(12);
     __syncthreads();
-    if (warp_id() == 0) {
-        const int ab = static_cast<int>(hist[WB]);
-        uint32_t cnt[P];
-        if (P == 2) {
-            const uint2 v = *reinterpret_cast<const uint2*>(hist + lane * 2);
-            cnt[0] = v.x;
-            cnt[1] = v.y;
-        } else {
+    AFX_MARK(13);
+    // Every warp resolves the window for itself from the same counters: nothing to broadcast.
+    constexpr int NW = NT / 32;
+    const int ab = __reduce_add_sync(0xFFFFFFFFu, lane < NW ? s->wtot[0][lane] : 0);
+    uint32_t cnt[P];
+    if (P == 2) {
+        const uint2 v = *reinterpret_cast<const uint2*>(hist + lane * 2);
+        cnt[0] = v.x;
+        cnt[1] = v.y;
+    } else {
 #pragma unroll
-            for (int q = 0; q < P / 4; ++q) {
-                const uint4 v = *reinterpret_cast<const uint4*>(hist + lane * P + q * 4);
-                cnt[4 * q] = v.x;
-                cnt[4 * q + 1] = v.y;
-                cnt[4 * q + 2] = v.z;
-                cnt[4 * q + 3] = v.w;
-            }
+        for (int q = 0; q < P / 4; ++q) {
+            const uint4 v = *reinterpret_cast<const uint4*>(hist + lane * P + q * 4);
+            cnt[4 * q] = v.x;
+            cnt[4 * q + 1] = v.y;
+            cnt[4 * q + 2] = v.z;
+            cnt[4 * q + 3] = v.w;
         }
-        int lane_sum = 0;
-#pragma unroll
-        for (int q = 0; q < P; ++q) lane_sum += static_cast<int>(cnt[q]);
-        int suf = lane_sum;  // inclusive suffix sums: higher lanes hold higher keys
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int n = __shfl_down_sync(0xFFFFFFFFu, suf, o);
-            if (lane + o < 32) suf += n;
-        }
-        const int inside = __shfl_sync(0xFFFFFFFFu, suf, 0);
-        const bool ok = ab < k && k <= ab + inside;
-        if (ok) {
-            int rem = k - ab;  // rank from the top inside the window
-            const uint32_t has = __ballot_sync(0xFFFFFFFFu, suf >= rem);
-            if (lane == 31 - __clz(static_cast<int>(has))) {
-                rem -= suf - lane_sum;
-                bool done = false;
-#pragma unroll
-                for (int q = P - 1; q >= 0; --q) {
-                    const int cq = static_cast<int>(cnt[q]);
-                    if (!done) {
-                        if (rem <= cq) {
-                            done = true;
-                            s->res[0] = lo + lane * P + q;
-                            s->res[1] = rem;
-                            s->res[2] = cq;
-                        } else {
-                            rem -= cq;
-                        }
-                    }
-                }
-            }
-        }
-        if (lane == 0) s->res[3] = ok ? 1 : 0;
     }
-    __syncthreads();
-    if (s->res[3] == 0) {
-        for (int i = threadIdx.x; i <= WB; i += NT) hist[i] = 0u;
+    int lane_sum = 0;
+#pragma unroll
+    for (int q = 0; q < P; ++q) lane_sum += static_cast<int>(cnt[q]);
+    int suf = lane_sum;  // inclusive suffix sums: higher lanes hold higher keys
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int n = __shfl_down_sync(0xFFFFFFFFu, suf, o);
+        if (lane + o < 32) suf += n;
+    }
+    const int inside = __shfl_sync(0xFFFFFFFFu, suf, 0);
+    if (!(ab < k && k <= ab + inside)) {  // same verdict in every warp
+        __syncthreads();                  // every warp has read the window
+        for (int i = threadIdx.x; i < WB; i += NT) hist[i] = 0u;
         __syncthreads();
         return false;
     }
-    thr = static_cast<uint32_t>(s->res[0]);
-    need_eq = s->res[1];
-    tot_eq = s->res[2];
+    int rem = k - ab;  // rank from the top inside the window
+    const uint32_t has = __ballot_sync(0xFFFFFFFFu, suf >= rem);
+    const int l_star = 31 - __clz(static_cast<int>(has));
+    int my_thr = 0, my_need = 0, my_tot = 0;
+    if (lane == l_star) {
+        rem -= suf - lane_sum;
+        bool done = false;
+#pragma unroll
+        for (int q = P - 1; q >= 0; --q) {
+            const int cq = static_cast<int>(cnt[q]);
+            if (!done) {
+                if (rem <= cq) {
+                    done = true;
+                    my_thr = lo + lane * P + q;
+                    my_need = rem;
+                    my_tot = cq;
+                } else {
+                    rem -= cq;
+                }
+            }
+        }
+        if (warp_id() == 0) s->res[0] = my_thr;  // for the caller that records the key
+    }
+    thr = static_cast<uint32_t>(__shfl_sync(0xFFFFFFFFu, my_thr, l_star));
+    need_eq = __shfl_sync(0xFFFFFFFFu, my_need, l_star);
+    tot_eq = __shfl_sync(0xFFFFFFFFu, my_tot, l_star);
     return true;
 }
 
@@ -411,6 +414,7 @@ __device__ __forceinline__ unsigned long long block_token_flags(const uint16_t* 
     int need_eq, tot_eq;
     if (!(single && hint != kNoKeyHint && block_kth_key_near<DT, NT>(xs, K, k, hint, hist, s, thr, need_eq, tot_eq)))
         block_kth_key<NT>(xs, K, k, hist, s, thr, need_eq, tot_eq);
+    AFX_MARK(8);
     // Channels above the k-th key are in; of those equal to it, the need_eq lowest ids.  One
     // pass over the thread's chunks, two keys per operation (swar_*), leaves two flag sets in
     // registers: keys greater than the k-th and keys equal to it.  A partial last chunk is
@@ -435,6 +439,7 @@ __device__ __forceinline__ unsigned long long block_token_flags(const uint16_t* 
         fe |= static_cast<unsigned long long>(ebyte) << (8 * (c - c_lo));
     }
     const int g = __popcll(fg), e_cnt = __popcll(fe);
+    AFX_MARK(9);
     int pre_e = 0;
     if (single) {
         int tot;
@@ -446,6 +451,7 @@ __device__ __forceinline__ unsigned long long block_token_flags(const uint16_t* 
         int tot;
         pre_e = block_prefix(e_cnt, s->wtot[1], tot);
     }
+    AFX_MARK(10);
     fl = fg;
     if (need_eq == tot_eq) {
         fl |= fe;
