@@ -330,10 +330,12 @@ def run_afx(args):
     N_gu = 2 * cfg["mlp"]
     y_dev = torch.empty((1, N_gu), dtype=torch.float32, device="cuda")
 
+    hint_slots = torch.zeros(len(layers), dtype=torch.int32, device="cuda")  # one per operator, as in the model
+
     def gu_pass():
-        for L in layers:
+        for i, L in enumerate(layers):
             afx.afx_select_gemv(L["w_gu"], cfg["dtype"], cfg["hidden"], N_gu, N_gu, x_dev, 1, afx.MODE_TOPK,
-                                k[2], 0.0, y_dev, 0, None, None, stream=st)
+                                k[2], 0.0, y_dev, 0, None, None, stream=st, kth_hint=hint_slots[i:i + 1])
 
     g2 = torch.cuda.CUDAGraph()
     with torch.cuda.stream(st):

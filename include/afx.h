@@ -113,11 +113,17 @@ afx_status afx_sparse_gemv(const void* Wt, int dtype, int K, int N, int64_t ldw,
  *   Wt, x, y, accumulate   as for afx_sparse_gemv;  mode, k, tau  as for afx_select_active.
  *   idx_out   DEVICE int32[K] or NULL: receives the active list.
  *   count_out DEVICE int32[1] or NULL: receives its length.
+ *   kth_hint  DEVICE int32[1] or NULL, read and rewritten by a top-k call with T == 1 and
+ *             0 < k < K: on return 0x10000 | the k-th largest magnitude key (the 16-bit pattern
+ *             with the sign cleared).  A value with bit 16 set that a call finds there is where
+ *             its search for the k-th key starts (cheap when the key lies within about 19 % of
+ *             it, e.g. the previous token's key for the same operator; the full search
+ *             otherwise); 0 means no hint.  The selected set never depends on it.
  * K * T * 2 bytes of x are read by every thread block (they stay in L2).
  */
 afx_status afx_select_gemv(const void* Wt, int dtype, int K, int N, int64_t ldw, const void* x, int T,
                            int mode, int k, float tau, float* y, int accumulate, int32_t* idx_out,
-                           int32_t* count_out, void* stream);
+                           int32_t* count_out, int32_t* kth_hint, void* stream);
 
 /* ------------------------------------------------------------------------------------------
  * Decoder layers: every linear operator of a Llama-shaped layer run as ONE kernel that

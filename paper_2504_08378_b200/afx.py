@@ -78,7 +78,7 @@ def lib() -> ctypes.CDLL:
         L.afx_sparse_gemv.argtypes = [c_void_p, c_int, c_int, c_int, c_int64, c_void_p, c_int,
                                       c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p]
         L.afx_select_gemv.argtypes = [c_void_p, c_int, c_int, c_int, c_int64, c_void_p, c_int, c_int, c_int,
-                                      c_float, c_void_p, c_int, c_void_p, c_void_p, c_void_p]
+                                      c_float, c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p]
         L.afx_model_create.argtypes = [ctypes.POINTER(ModelDesc), ctypes.POINTER(LayerDesc),
                                        ctypes.POINTER(c_void_p)]
         L.afx_model_destroy.argtypes = [c_void_p]
@@ -161,11 +161,11 @@ def afx_sparse_gemv(Wt, dtype, K: int, N: int, ldw: int, x, T: int, idx, count, 
 
 
 def afx_select_gemv(Wt, dtype, K: int, N: int, ldw: int, x, T: int, mode: int, k: int, tau: float, y,
-                    accumulate: int, idx_out=None, count_out=None, stream=None):
+                    accumulate: int, idx_out=None, count_out=None, stream=None, kth_hint=None):
     _check("afx_select_gemv",
            lib().afx_select_gemv(_ptr(Wt), _dt(dtype), int(K), int(N), int(ldw), _ptr(x), int(T), int(mode),
                                  int(k), float(tau), _ptr(y), int(accumulate), _ptr(idx_out), _ptr(count_out),
-                                 _stream(stream)))
+                                 _ptr(kth_hint), _stream(stream)))
 
 
 def afx_model_create(desc: ModelDesc, layers) -> int:

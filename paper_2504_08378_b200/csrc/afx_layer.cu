@@ -446,7 +446,7 @@ extern "C" afx_status afx_mlp_block(afx_model* m, int layer, afx_state* s, const
 
 extern "C" afx_status afx_select_gemv(const void* Wt, int dtype, int K, int N, int64_t ldw, const void* x, int T,
                                       int mode, int k, float tau, float* y, int accumulate, int32_t* idx_out,
-                                      int32_t* count_out, void* stream) {
+                                      int32_t* count_out, int32_t* kth_hint, void* stream) {
     using namespace afx;
     if (Wt == nullptr || x == nullptr || y == nullptr) return AFX_ERR_INVALID_ARG;
     if (K <= 0 || N <= 0 || T < 1 || T > AFX_MAX_T || ldw < N) return AFX_ERR_INVALID_ARG;
@@ -457,7 +457,7 @@ extern "C" afx_status afx_select_gemv(const void* Wt, int dtype, int K, int N, i
     if (mode == AFX_MODE_THRESHOLD && tau != tau) return AFX_ERR_INVALID_ARG;
     if ((N & 7) != 0 || (ldw & 7) != 0 || !aligned16(Wt) || !aligned16(y) ||
         (reinterpret_cast<uintptr_t>(x) & 1u) != 0 || (reinterpret_cast<uintptr_t>(idx_out) & 3u) != 0 ||
-        (reinterpret_cast<uintptr_t>(count_out) & 3u) != 0)
+        (reinterpret_cast<uintptr_t>(count_out) & 3u) != 0 || (reinterpret_cast<uintptr_t>(kth_hint) & 3u) != 0)
         return AFX_ERR_ALIGNMENT;
     if ((N + 63) / 64 > 65535) return AFX_ERR_CAPACITY;
     FusedArgs a = {};
@@ -473,6 +473,7 @@ extern "C" afx_status afx_select_gemv(const void* Wt, int dtype, int K, int N, i
     a.ep = {y, nullptr, N};
     a.idx_out = idx_out;
     a.count_out = count_out;
+    a.kth_slot = kth_hint;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     return accumulate ? launch_fused<IN_X, EP_ACCUM>(dtype, a, st) : launch_fused<IN_X, EP_STORE>(dtype, a, st);
 }

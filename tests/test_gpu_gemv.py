@@ -156,3 +156,30 @@ def test_select_gemv_equals_select_then_gemv(dt, K, N, T):
         n = int(cnt_d.item())
         assert n == want.size and np.array_equal(idx_d.cpu().numpy()[:n], want)
         assert rel_err(y.cpu().numpy(), oracle.sparse_gemv(Wt, dt, N, x, want)) <= TOL
+
+
+@pytest.mark.parametrize("dt", ["f16", "bf16"])
+def test_select_gemv_hint_slot(dt):
+    """kth_hint: the call records 0x10000 | k-th key; whatever it finds there first (nothing, the
+    exact key, a near or far key, garbage) the list and y are the same."""
+    K, N, T = 4096, 1024 + 24, 1
+    k = synth.keep_count(K, 50)
+    Wt = synth.weight(221, 1, K, N, dt)
+    x = synth.laplace_bits(222, 2, (T, K), dt)
+    W, xd = dev_bits(Wt), dev_bits(x)
+    want = oracle.select_active(x, dt, afx.MODE_TOPK, k=k)
+    y_ref = oracle.sparse_gemv(Wt, dt, N, x, want)
+    keys = np.sort(x.reshape(-1).astype(np.int64) & 0x7FFF)
+    exact = int(keys[K - k])
+    slot = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for preset in (0, None, 0x10000 | (exact + 3), 0x10000 | max(0, exact - 2000), 0x10000 | 0x7FFF, 0x7FFF, -1):
+        if preset is not None:  # None: keep what the previous call recorded (the exact key)
+            slot.fill_(preset)
+        idx_d = torch.full((K,), -3, dtype=torch.int32, device="cuda")
+        cnt_d = torch.full((1,), -3, dtype=torch.int32, device="cuda")
+        y = torch.full((T, N), float("nan"), dtype=torch.float32, device="cuda")
+        afx.afx_select_gemv(W, dt, K, N, N, xd, T, afx.MODE_TOPK, k, 0.0, y, 0, idx_d, cnt_d, kth_hint=slot)
+        torch.cuda.synchronize()
+        assert int(slot.item()) == 0x10000 | exact, preset
+        assert int(cnt_d.item()) == k and np.array_equal(idx_d.cpu().numpy()[:k], want), preset
+        assert rel_err(y.cpu().numpy(), y_ref) <= TOL, preset
