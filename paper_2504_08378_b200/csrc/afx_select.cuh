@@ -299,7 +299,7 @@ __device__ __forceinline__ bool block_kth_key_near(const uint16_t* xs, int K, in
         if (lane + o < 32) suf += n;
     }
     const int inside = __shfl_sync(0xFFFFFFFFu, suf, 0);
-    if (!(ab < k && k <= ab + inside)) {  // same verdict in every warp
+    if (!(ab < k && k <= ab + inside)) {  // same outcome in every warp
         __syncthreads();                  // every warp has read the window
         for (int i = threadIdx.x; i < WB; i += NT) hist[i] = 0u;
         __syncthreads();
