@@ -147,12 +147,18 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
                 ss = fmaf(v.w, v.w, ss);
             }
             ss = warp_sum(ss);
-            __syncthreads();
+            if (t > 0) __syncthreads();  // the previous token's sums have been read
             if (lane == 0) red16[warp] = ss;
             __syncthreads();
-            float tot = 0.0f;
+            float tot = 0.0f;  // the 16 warp sums in warp order, read four at a time
 #pragma unroll
-            for (int w = 0; w < kGemvWarps; ++w) tot += red16[w];
+            for (int w = 0; w < kGemvWarps; w += 4) {
+                const float4 v = *reinterpret_cast<const float4*>(red16 + w);
+                tot += v.x;
+                tot += v.y;
+                tot += v.z;
+                tot += v.w;
+            }
             const float inv = 1.0f / sqrtf(tot / static_cast<float>(K) + a.eps);
             const float4* gq = reinterpret_cast<const float4*>(a.gain);
             auto emit = [&](int c, const float4& v, const float4& g) {

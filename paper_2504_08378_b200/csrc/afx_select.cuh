@@ -30,7 +30,7 @@ constexpr size_t kKeyHistBytes = static_cast<size_t>(kKeyHistWords) * 4;
 struct SelectScratch {
     int wtot[4][32];  // per-warp totals for the ordered scans
     int res[4];       // broadcast of the k-th key search
-    int hist[256];    // large-K path; the fused operators borrow it for the norm's reduction
+    __align__(16) int hist[256];  // large-K path; the fused operators borrow it for the norm's reduction
     int scan[33];
 };
 
