@@ -19,6 +19,15 @@
  *   - An active list is `idx[0..*count)`, int32 channel ids in strictly ascending order,
  *     with the count in DEVICE memory so that no host round trip sits between selection
  *     and the GEMV.
+ *   - `dev_status` (where an entry point has it) is a DEVICE int32 or NULL.  Lists and counts
+ *     that a kernel reads from caller memory cannot be validated on the host, so the kernels
+ *     check them: a count outside [0, K] is clamped (AFX_ERR_CAPACITY), a channel id outside
+ *     [0, K) is skipped (AFX_ERR_INVALID_ARG), a negative cache slot is skipped
+ *     (AFX_ERR_CAPACITY: the cache ran out of staging rows).  Nothing traps and no address
+ *     outside the caller's buffers is formed; the first such event stores its code into
+ *     *dev_status if that still holds 0.  The library never clears the word.
+ *   - Nothing in the paper prescribes this interface; where an entry point or a parameter is
+ *     this library's own device rather than the paper's, its comment says so.
  */
 #ifndef AFX_H
 #define AFX_H
@@ -38,7 +47,8 @@ typedef int32_t afx_status;
 #define AFX_ERR_CAPACITY 3    /* a caller-provided buffer or a fixed limit is too small */
 #define AFX_ERR_UNSUPPORTED 4 /* unknown dtype or mode */
 #define AFX_ERR_CUDA 5        /* the CUDA runtime refused a launch or a query */
-#define AFX_ERR_TIMEOUT 6     /* a bounded device-side wait gave up (reported via a status word) */
+#define AFX_ERR_TIMEOUT 6     /* reserved: a bounded device-side wait gave up.  No kernel of this */
+                              /* version waits on a flag, so nothing returns or stores it.        */
 
 #define AFX_F16 0
 #define AFX_BF16 1
@@ -53,6 +63,15 @@ afx_status afx_version(int* major, int* minor);
 
 /* Static, human-readable name of a status code (HOST string, never NULL). */
 const char* afx_status_string(afx_status s);
+
+/*
+ * Bytes of DEVICE scratch memory the entry points below need for operators of up to K_max
+ * channels, N_max outputs and T_max tokens: always 0.  Partial sums meet in shared memory and
+ * in the distributed shared memory of a thread-block cluster, and the selection runs inside
+ * the consuming kernel, so no call takes a workspace pointer.  (Interface bookkeeping; the
+ * paper has no counterpart.)
+ */
+size_t afx_workspace_bytes(int K_max, int N_max, int T_max);
 
 /*
  * Active-channel selection ("Top-K" operation T of the swapping pipeline, Sec. 4; the
@@ -78,11 +97,12 @@ afx_status afx_select_active(const void* x, int dtype, int K, int T, int mode, i
  * Cross-layer bookkeeping (Sec. 3: an earlier layer's activation predicts this layer's
  * active set; what the prediction missed is fetched on demand).  A = idxA[0..*cntA) is the
  * actual set, P the predicted set given as a bitmap.  Writes miss = A \ P ascending
- * (capacity K), *miss_count = |A \ P| and *hit_count = |A & P|.  All pointers DEVICE.
+ * (capacity K), *miss_count = |A \ P| and *hit_count = |A & P|.  All pointers DEVICE, 4-byte
+ * aligned.  An entry of A outside [0, K) counts as neither (see dev_status above).
  */
 afx_status afx_diff_active(const int32_t* idxA, const int32_t* cntA, const uint32_t* bitmapP,
                            int K, int32_t* miss, int32_t* miss_count, int32_t* hit_count,
-                           void* stream);
+                           int32_t* dev_status, void* stream);
 
 /*
  * Sparse GEMV over the active channels (operation C of the pipeline; Sec. 2.1: only the
@@ -96,19 +116,25 @@ afx_status afx_diff_active(const int32_t* idxA, const int32_t* cntA, const uint3
  *
  *   Wt        DEVICE, channel-contiguous weights (see the conventions above).
  *   x         DEVICE, [T][K] 16-bit floats; every token uses the whole list.
- *   idx,count DEVICE; entries must lie in [0,K) (not checked on the device).
- *   slot      DEVICE int32[*count] or NULL.
+ *   idx,count DEVICE; an entry outside [0,K) contributes nothing (see dev_status above).
+ *   slot      DEVICE int32[*count] or NULL; a negative slot contributes nothing (afx_cache_fetch
+ *             writes -1 for a channel it could not place), an upper bound is the caller's to keep
+ *             (the kernel does not know how many rows Wt has when it is a cache).
  *   y         DEVICE, [T][N] fp32, 16-byte aligned.  accumulate = 0 overwrites, 1 adds.
+ *   dev_status DEVICE int32 or NULL.
  * Needs no scratch memory.  N <= 4 194 240.
  */
 afx_status afx_sparse_gemv(const void* Wt, int dtype, int K, int N, int64_t ldw, const void* x,
                            int T, const int32_t* idx, const int32_t* count, const int32_t* slot,
-                           float* y, int accumulate, void* stream);
+                           float* y, int accumulate, int32_t* dev_status, void* stream);
 
 /*
  * Selection and sparse GEMV in ONE kernel (the T and C operations of Sec. 4 back to back):
  * the result equals afx_select_active followed by afx_sparse_gemv on the same arguments,
- * without the list's round trip through global memory between two launches.
+ * without the list's round trip through global memory between two launches.  The paper runs T
+ * and C as separate pipeline stages; fusing them, and the `kth_hint` slot, are this library's
+ * own design for a GPU (the hint is an accelerator only: the paper's thresholds are calibrated
+ * offline, here the exact top-k search merely starts near the previous answer).
  *
  *   Wt, x, y, accumulate   as for afx_sparse_gemv;  mode, k, tau  as for afx_select_active.
  *   idx_out   DEVICE int32[K] or NULL: receives the active list.
@@ -187,6 +213,8 @@ afx_status afx_model_create(const afx_model_desc* desc, const afx_layer_desc* la
 afx_status afx_model_destroy(afx_model* model);
 
 /*
+ * (The state object and its accessors are this library's own plumbing; the paper has no
+ * counterpart.)
  * Per-sequence working set for T token streams decoded together (1 <= T <= AFX_MAX_T): the
  * fp32 residual h[T][hidden], the operators' intermediate vectors, the current and predicted
  * active sets of the four operator inputs, and per-layer counters.  The caller allocates
@@ -223,6 +251,19 @@ afx_status afx_state_buffer(const afx_state* state, int which, int op, void** pt
  * Layers must be stepped in order 0 .. n_layers-1 when cross-layer prediction is on.
  */
 afx_status afx_layer_step(afx_model* model, int layer, afx_state* state, int pos, void* stream);
+
+/*
+ * ONE of the five kernels of afx_layer_step, on whatever the state holds (afx_layer_step is
+ * exactly the five calls in order).  For per-operator timing and profiling of the launches a
+ * decode step really makes -- the same kernel instantiation, launch shape and side outputs;
+ * this library's own addition, the paper has no counterpart.
+ */
+#define AFX_STEP_QKV 0
+#define AFX_STEP_ATTN 1
+#define AFX_STEP_O 2
+#define AFX_STEP_GU 3
+#define AFX_STEP_DOWN 4
+afx_status afx_layer_kernel(afx_model* model, int layer, afx_state* state, int pos, int which, void* stream);
 
 /*
  * The MLP block alone on a given (already normalised) input: y = W_down(silu(W_gate x) * W_up x)
@@ -288,13 +329,17 @@ afx_status afx_cache_install(afx_cache* cache, const int32_t* host_channels, int
 
 /*
  * One step.  idx / count: DEVICE active list (ascending; as afx_select_active writes it).
- * slot_out: DEVICE int32[K]; entry c receives the row of idx[c] in `slots`.  stats: DEVICE
- * afx_cache_stats or NULL.  Two kernels on `stream`: the policy (one thread block; the
- * victims are ordered by a bitonic sort of (count, channel) keys) and the copy of the missed
- * channels (128-bit loads from the mapped host memory).  No host synchronisation.
+ * slot_out: DEVICE int32[K]; entry c receives the row of idx[c] in `slots` (-1 for a transient
+ * that found no staging row, and for an entry outside [0, K), which takes no part in the
+ * step).  stats: DEVICE afx_cache_stats or NULL.  dev_status: DEVICE int32 or NULL (see the
+ * conventions at the top; staging overflow stores AFX_ERR_CAPACITY, and afx_sparse_gemv then
+ * leaves the unplaced channels out instead of reading a row that does not exist).  Two
+ * kernels on `stream`: the policy (one thread block; the victims are ordered by a bitonic
+ * sort of (count, channel) keys) and the copy of the missed channels (128-bit loads from the
+ * mapped host memory).  No host synchronisation.
  */
 afx_status afx_cache_fetch(afx_cache* cache, const int32_t* idx, const int32_t* count, int32_t* slot_out,
-                           afx_cache_stats* stats, void* stream);
+                           afx_cache_stats* stats, int32_t* dev_status, void* stream);
 
 /* Copies the tables to HOST arrays for inspection (either may be NULL): slot_of[K] (-1 = not
  * cached), usage[K].  Synchronises the stream. */
@@ -319,8 +364,10 @@ afx_status afx_cache_snapshot(afx_cache* cache, int32_t* host_slot_of, uint32_t*
  *           overwritten.  mode, k_*, tau_* as for afx_select_active, per operator.
  * hidden and mlp are multiples of 8; hidden <= 32768; mlp > AFX_NOALLOC_MAX_MLP returns
  * AFX_ERR_CAPACITY and launches nothing.
- * The first call on a device looks up the array's device address (with that device current);
- * make that first call outside any stream capture.  All calls on a device share the array and
+ * The first call on a device looks up the array's device address (with that device current)
+ * and keeps it for the life of the process (it does not survive cudaDeviceReset); make that
+ * first call outside any stream capture -- a first call on a capturing stream returns
+ * AFX_ERR_INVALID_ARG and launches nothing.  All calls on a device share the array and
  * it keeps the previous call's contents (nothing in it has to start from zero: each call
  * rewrites the T * mlp values it reads): two calls whose kernels overlap on the GPU -- different
  * streams, or graphs replayed concurrently -- race on it; serialise them.

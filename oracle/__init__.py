@@ -57,6 +57,11 @@ def threads() -> int:
     return int(lib().afxo_threads())
 
 
+def set_threads(n: int) -> None:
+    """Caps the oracle's worker threads (for a one-core timing); results do not depend on it."""
+    lib().afxo_set_threads(int(n))
+
+
 def decode(bits, dtype: str) -> np.ndarray:
     """fp64 values of 16-bit patterns."""
     bits = _u16(bits)

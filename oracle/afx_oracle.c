@@ -276,6 +276,18 @@ int afxo_threads(void)
 #endif
 }
 
+/* Caps the threads the row-parallel loops may use (timing the oracle on one core); no effect
+ * on any result: every output row is summed by one thread in the same order. */
+void afxo_set_threads(int n)
+{
+#ifdef _OPENMP
+    if (n >= 1)
+        omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
 /* ---------------------------------------------------------------- decoder-layer glue */
 
 /* out[t][j] = round_dtype( h[t][j] / sqrt(mean_j h^2 + eps) * g[j] ) */

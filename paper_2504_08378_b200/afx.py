@@ -16,6 +16,7 @@ F16, BF16 = 0, 1
 OP_QKV, OP_O, OP_GU, OP_DOWN = 0, 1, 2, 3
 XL_OFF, XL_BOOKKEEP, XL_REUSE = 0, 1, 2
 BUF_H, BUF_QKV, BUF_ATTN, BUF_HM, BUF_XNORM, BUF_IDX, BUF_MISS, BUF_STATS = range(8)
+STEP_QKV, STEP_ATTN, STEP_O, STEP_GU, STEP_DOWN = range(5)
 MODE_TOPK, MODE_THRESHOLD = 0, 1
 MAX_T = 8
 DTYPES = {"f16": F16, "bf16": BF16}
@@ -73,10 +74,12 @@ def lib() -> ctypes.CDLL:
         L.afx_status_string.argtypes = [c_int32]
         L.afx_select_active.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_int, c_float,
                                         c_void_p, c_void_p, c_void_p, c_void_p]
+        L.afx_workspace_bytes.restype = c_size_t
+        L.afx_workspace_bytes.argtypes = [c_int, c_int, c_int]
         L.afx_diff_active.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p,
-                                      c_void_p, c_void_p]
+                                      c_void_p, c_void_p, c_void_p]
         L.afx_sparse_gemv.argtypes = [c_void_p, c_int, c_int, c_int, c_int64, c_void_p, c_int,
-                                      c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p]
+                                      c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p]
         L.afx_select_gemv.argtypes = [c_void_p, c_int, c_int, c_int, c_int64, c_void_p, c_int, c_int, c_int,
                                       c_float, c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p]
         L.afx_model_create.argtypes = [ctypes.POINTER(ModelDesc), ctypes.POINTER(LayerDesc),
@@ -90,12 +93,13 @@ def lib() -> ctypes.CDLL:
         L.afx_state_buffer.argtypes = [c_void_p, c_int, c_int, ctypes.POINTER(c_void_p),
                                        ctypes.POINTER(c_size_t)]
         L.afx_layer_step.argtypes = [c_void_p, c_int, c_void_p, c_int, c_void_p]
+        L.afx_layer_kernel.argtypes = [c_void_p, c_int, c_void_p, c_int, c_int, c_void_p]
         L.afx_mlp_block.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p]
         L.afx_cache_create.argtypes = [ctypes.POINTER(CacheDesc), ctypes.POINTER(c_void_p)]
         L.afx_cache_destroy.argtypes = [c_void_p]
         L.afx_cache_reset.argtypes = [c_void_p, c_void_p]
         L.afx_cache_install.argtypes = [c_void_p, c_void_p, c_int, c_void_p]
-        L.afx_cache_fetch.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+        L.afx_cache_fetch.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
         L.afx_cache_snapshot.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p]
         L.afx_mlp_block_noalloc.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_void_p, c_int, c_int, c_int,
                                             c_float, c_int, c_float, c_void_p, c_void_p]
@@ -146,18 +150,22 @@ def afx_select_active(x, dtype, K: int, T: int, mode: int, k: int, tau: float, i
                                    _ptr(idx), _ptr(count), _ptr(bitmap), _stream(stream)))
 
 
-def afx_diff_active(idxA, cntA, bitmapP, K: int, miss, miss_count, hit_count, stream=None):
+def afx_workspace_bytes(K_max: int, N_max: int, T_max: int) -> int:
+    return int(lib().afx_workspace_bytes(int(K_max), int(N_max), int(T_max)))
+
+
+def afx_diff_active(idxA, cntA, bitmapP, K: int, miss, miss_count, hit_count, stream=None, dev_status=None):
     _check("afx_diff_active",
            lib().afx_diff_active(_ptr(idxA), _ptr(cntA), _ptr(bitmapP), int(K), _ptr(miss),
-                                 _ptr(miss_count), _ptr(hit_count), _stream(stream)))
+                                 _ptr(miss_count), _ptr(hit_count), _ptr(dev_status), _stream(stream)))
 
 
 def afx_sparse_gemv(Wt, dtype, K: int, N: int, ldw: int, x, T: int, idx, count, slot, y,
-                    accumulate: int, stream=None):
+                    accumulate: int, stream=None, dev_status=None):
     _check("afx_sparse_gemv",
            lib().afx_sparse_gemv(_ptr(Wt), _dt(dtype), int(K), int(N), int(ldw), _ptr(x), int(T),
                                  _ptr(idx), _ptr(count), _ptr(slot), _ptr(y), int(accumulate),
-                                 _stream(stream)))
+                                 _ptr(dev_status), _stream(stream)))
 
 
 def afx_select_gemv(Wt, dtype, K: int, N: int, ldw: int, x, T: int, mode: int, k: int, tau: float, y,
@@ -206,6 +214,10 @@ def afx_layer_step(model: int, layer: int, state: int, pos: int, stream=None):
     _check("afx_layer_step", lib().afx_layer_step(model, int(layer), state, int(pos), _stream(stream)))
 
 
+def afx_layer_kernel(model: int, layer: int, state: int, pos: int, which: int, stream=None):
+    _check("afx_layer_kernel", lib().afx_layer_kernel(model, int(layer), state, int(pos), int(which), _stream(stream)))
+
+
 def afx_mlp_block(model: int, layer: int, state: int, x, y, stream=None):
     _check("afx_mlp_block", lib().afx_mlp_block(model, int(layer), state, _ptr(x), _ptr(y), _stream(stream)))
 
@@ -241,9 +253,10 @@ def afx_cache_install(cache: int, channels, stream=None):
     _check("afx_cache_install", lib().afx_cache_install(cache, arr, len(channels), _stream(stream)))
 
 
-def afx_cache_fetch(cache: int, idx, count, slot_out, stats=None, stream=None):
+def afx_cache_fetch(cache: int, idx, count, slot_out, stats=None, stream=None, dev_status=None):
     _check("afx_cache_fetch",
-           lib().afx_cache_fetch(cache, _ptr(idx), _ptr(count), _ptr(slot_out), _ptr(stats), _stream(stream)))
+           lib().afx_cache_fetch(cache, _ptr(idx), _ptr(count), _ptr(slot_out), _ptr(stats), _ptr(dev_status),
+                                 _stream(stream)))
 
 
 def afx_cache_snapshot(cache: int, K: int, stream=None):

@@ -81,12 +81,12 @@ __device__ __forceinline__ void attention_block(const AttnArgs& a, AttnSmem* sm)
     const uint32_t half_mask = 0xFFFFu << (16 * half);  // the two halves of a warp work on different keys
 
     AFX_MARK(0);
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     uint16_t* kc = a.k_cache + static_cast<size_t>(t) * a.max_seq * a.kv_heads * kHeadDim;
     uint16_t* vc = a.v_cache + static_cast<size_t>(t) * a.max_seq * a.kv_heads * kHeadDim;
     // With one query head per kv head the registers allow it: the past rows of this half
-    // warp's first batch do not depend on the kernel that is still running (they were written
-    // by earlier tokens), so they are requested before the wait for q, k, v.
+    // warp's first batch were written by earlier tokens' attention kernels -- at least one
+    // layer step (five grids) back, so complete by the ordering rule stated in fused_op_block
+    // -- and are requested before the wait for q, k, v.
     constexpr int U = REP == 1 ? 2 * kAttnUnroll : kAttnUnroll;
     constexpr bool kEarly = REP == 1;
     uint4 kraw[U], vraw[U];
@@ -103,6 +103,7 @@ __device__ __forceinline__ void attention_block(const AttnArgs& a, AttnSmem* sm)
         }
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // only after the wait (see fused_op_block)
     AFX_MARK(1);
 
     const float* row = a.qkv + static_cast<size_t>(t) * a.n_qkv;

@@ -44,12 +44,13 @@ __device__ __forceinline__ void owned_range(int n, int& lo, int& hi) {
 
 __global__ void __launch_bounds__(kCacheThreads, 1)
 cache_policy_kernel(CacheTables tb, const int32_t* __restrict__ idx, const int32_t* __restrict__ count,
-                    int32_t* __restrict__ slot_out, afx_cache_stats* __restrict__ stats, int N) {
+                    int32_t* __restrict__ slot_out, afx_cache_stats* __restrict__ stats, int N,
+                    int32_t* __restrict__ status) {
     extern __shared__ __align__(16) unsigned char dyn[];
     __shared__ int scan[4][32];
     __shared__ int s_mfreq[kCacheThreads];
     __shared__ int s_assign[kCacheThreads];
-    __shared__ int s_vp, s_nt;
+    __shared__ int s_vp, s_nt, s_bad;
     const int K = tb.K, C = tb.C;
     const int nwords = (K + 31) >> 5;
     uint32_t* active = reinterpret_cast<uint32_t*>(dyn);
@@ -58,17 +59,28 @@ cache_policy_kernel(CacheTables tb, const int32_t* __restrict__ idx, const int32
                                    : tb.keys;
     const int tid = threadIdx.x;
     int n = *count;
-    n = max(0, min(n, K));
+    if (n < 0 || n > K) {
+        if (tid == 0) report_status(status, AFX_ERR_CAPACITY);
+        n = max(0, min(n, K));
+    }
+    // a list entry outside [0, K) takes no part in the step: no count, no slot (-1), neither a
+    // hit nor a miss; the status word reports it
+    auto valid = [&](int j) { return static_cast<unsigned>(j) < static_cast<unsigned>(K); };
 
     // 1. activity bitmap and usage counts
     for (int w = tid; w < nwords; w += blockDim.x) active[w] = 0u;
     if (tid == 0) {
         s_vp = 0;
         s_nt = 0;
+        s_bad = 0;
     }
     __syncthreads();
     for (int c = tid; c < n; c += blockDim.x) {
         const int j = idx[c];
+        if (!valid(j)) {
+            atomicAdd(&s_bad, 1);
+            continue;
+        }
         atomicOr(&active[j >> 5], 1u << (j & 31));
         tb.usage[j] += 1u;  // list entries are distinct channels
     }
@@ -78,12 +90,13 @@ cache_policy_kernel(CacheTables tb, const int32_t* __restrict__ idx, const int32
     int lo, hi;
     owned_range(n, lo, hi);
     int mine = 0;
-    for (int c = lo; c < hi; ++c) mine += tb.slot_of[idx[c]] < 0;
+    for (int c = lo; c < hi; ++c) mine += valid(idx[c]) && tb.slot_of[idx[c]] < 0;
     int n_miss;
     int at = block_prefix(mine, scan[0], n_miss);
     for (int c = lo; c < hi; ++c) {
-        const int s = tb.slot_of[idx[c]];
-        if (s < 0)
+        const int j = idx[c];
+        const int s = valid(j) ? tb.slot_of[j] : -1;
+        if (valid(j) && s < 0)
             tb.miss_pos[at++] = c;
         else
             slot_out[c] = s;
@@ -186,10 +199,12 @@ cache_policy_kernel(CacheTables tb, const int32_t* __restrict__ idx, const int32
     }
     if (tid == 0) {
         *tb.n_fetch = n_miss;
+        const int nt = s_nt;
+        const int over = max(0, nt - tb.staging_rows);
+        if (s_bad > 0) report_status(status, AFX_ERR_INVALID_ARG);
+        if (over > 0) report_status(status, AFX_ERR_CAPACITY);
         if (stats != nullptr) {
-            const int nt = s_nt;
-            const int over = max(0, nt - tb.staging_rows);
-            stats->hits = n - n_miss;
+            stats->hits = n - n_miss - s_bad;
             stats->misses = n_miss;
             stats->transients = nt;
             stats->overflow = over;
@@ -340,15 +355,16 @@ extern "C" afx_status afx_cache_install(afx_cache* cache, const int32_t* host_ch
 }
 
 extern "C" afx_status afx_cache_fetch(afx_cache* cache, const int32_t* idx, const int32_t* count, int32_t* slot_out,
-                                      afx_cache_stats* stats, void* stream) {
+                                      afx_cache_stats* stats, int32_t* dev_status, void* stream) {
     using namespace afx;
     if (cache == nullptr || idx == nullptr || count == nullptr || slot_out == nullptr) return AFX_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(idx) & 3u) || (reinterpret_cast<uintptr_t>(count) & 3u) ||
-        (reinterpret_cast<uintptr_t>(slot_out) & 3u) || (reinterpret_cast<uintptr_t>(stats) & 7u))
+        (reinterpret_cast<uintptr_t>(slot_out) & 3u) || (reinterpret_cast<uintptr_t>(stats) & 7u) ||
+        (reinterpret_cast<uintptr_t>(dev_status) & 3u))
         return AFX_ERR_ALIGNMENT;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cache_policy_kernel<<<1, kCacheThreads, cache->policy_smem, st>>>(cache->tb, idx, count, slot_out, stats,
-                                                                       cache->d.N);
+                                                                       cache->d.N, dev_status);
     if (cudaGetLastError() != cudaSuccess) return AFX_ERR_CUDA;
     const int blocks = 4 * (sm_count() > 0 ? sm_count() : 148);
     cache_copy_kernel<<<blocks, kCopyThreads, 0, st>>>(

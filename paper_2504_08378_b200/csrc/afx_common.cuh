@@ -7,31 +7,10 @@
 
 #include "afx.h"
 
-// Stage marks for kernel timing studies: compiled out unless AFX_TRACE is defined, in which
-// case thread 0 of every block stores the SM clock of mark i (0..14) into afx_trace_buf, in
-// one of five regions told apart by the launch shape (256-thread blocks; 5-, 3- and other
-// cluster widths, the last split by dynamic shared memory above / below 80 KB), slots 15 and 14 of a block holding the global nanosecond timer and the SM
-// id at its mark 0.
+// Stage marks for kernel timing studies: empty unless the library is built with AFX_TRACE, in
+// which case afx_trace.cuh supplies the recording form.
 #ifdef AFX_TRACE
-extern __device__ long long afx_trace_buf[];
-#define AFX_MARK(i)                                                                                   \
-    do {                                                                                              \
-        if (threadIdx.x == 0) {                                                                       \
-            unsigned dyn_;                                                                            \
-            asm volatile("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn_));                            \
-            const int region_ = blockDim.x == 256 ? 0 : (gridDim.x == 5 ? 1 : (gridDim.x == 3 ? 2 : (dyn_ > 80000u ? 3 : 4))); \
-            long long* slot_ = afx_trace_buf + (region_ * 512 + (blockIdx.y * gridDim.x + blockIdx.x) % 512) * 16; \
-            slot_[(i)] = clock64();                                                                   \
-            if ((i) == 0) {                                                                           \
-                unsigned long long ns_;                                                               \
-                asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns_));                               \
-                slot_[15] = static_cast<long long>(ns_);                                              \
-                unsigned sm_;                                                                         \
-                asm volatile("mov.u32 %0, %%smid;" : "=r"(sm_));                                      \
-                slot_[14] = static_cast<long long>(sm_);                                              \
-            }                                                                                         \
-        }                                                                                             \
-    } while (0)
+#include "afx_trace.cuh"
 #else
 #define AFX_MARK(i) \
     do {            \
@@ -140,6 +119,14 @@ __device__ __forceinline__ int block_exclusive_over_warps(int warp_total, int* s
     }
     __syncthreads();
     return scratch[warp_id()];
+}
+
+// ---- device status word ----------------------------------------------------------------
+
+// Records the first problem a kernel met in caller-provided data (a list entry or a count out
+// of range): the word keeps the first non-zero code until the caller clears it.
+__device__ __forceinline__ void report_status(int32_t* status, int32_t code) {
+    if (status != nullptr) atomicCAS(status, 0, code);
 }
 
 // ---- host side -----------------------------------------------------------------------

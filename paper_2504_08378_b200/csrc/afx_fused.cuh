@@ -70,10 +70,7 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
     const int S = gridDim.x, s = blockIdx.x, tile = blockIdx.y;
     const int T = a.T, K = a.K;
     const bool side = a.side_cluster != 0 && blockIdx.y == gridDim.y - 1;  // the cluster without a tile
-    if (side && blockIdx.x != 0) {
-        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-        return;
-    }
+    if (side && blockIdx.x != 0) return;  // (a block that has left no longer holds back the next grid)
     // writes the side outputs: block 0 of the side cluster, else block (0,0) next to its GEMV work
     const bool scribe = a.side_cluster != 0 ? side : (blockIdx.x == 0 && blockIdx.y == 0);
     const int nwords = (K + 31) >> 5;
@@ -91,7 +88,12 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
     if (!side) cluster_arrive();  // the side cluster never meets
     if (topk) block_clear_key_hist<kGemvThreads>(hist);  // does not depend on the previous kernel
 
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // Ordering rule of every kernel of this library: a grid lets its successor be scheduled
+    // only AFTER its own dependency wait.  When a grid runs its prologue, its predecessor has
+    // therefore passed its wait, i.e. the grid before that one is complete: whatever is read
+    // before the wait below must have been written at least two grids earlier (weights and
+    // gains: never; the search hint and the predicted set: by the same operator of an earlier
+    // token or layer, at least five grids back).
     // the norm's gains are weights: they can be on their way before the wait for h
     constexpr int NH = 4;  // float4 pieces of h (and of the gain) a thread keeps in registers
     float4 gv[NH];
@@ -102,16 +104,17 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
             gv[i] = c < (K >> 2) ? reinterpret_cast<const float4*>(a.gain)[c] : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
         }
     }
-    // the hint was written by an earlier token's launch of this operator, not by the kernel
-    // waited for below (a launch that reads the value its own scribe block has just rewritten
-    // only gets a better hint: the selection's result does not depend on it)
+    // the hint was written by an earlier token's launch of this operator (a launch that reads
+    // the value its own scribe block has just rewritten only gets a better hint: the
+    // selection's result does not depend on it)
     uint32_t hint = kNoKeyHint;
     if (topk && T == 1 && a.kth_slot != nullptr) {
         const uint32_t v = static_cast<uint32_t>(__ldcg(a.kth_slot));
         if (v & 0x10000u) hint = v & 0x7FFFu;
     }
-    // likewise the predicted set this selection is compared with: the predictor layer wrote it
-    // several kernels ago (byte v = the flags of the v-th chunk this thread owns, like `fl`)
+    // likewise the predicted set this selection is compared with: the same operator of the
+    // predictor layer wrote it, at least one layer (five grids) ago (byte v = the flags of the
+    // v-th chunk this thread owns, like `fl`)
     unsigned long long pm = 0ull;
     if (scribe && own && a.bitmap_pred != nullptr) {
         int q_lo, q_hi;
@@ -120,6 +123,7 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
         for (int c = q_lo; c < q_hi; ++c) pm |= static_cast<unsigned long long>(__ldcg(pred + c)) << (8 * (c - q_lo));
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     AFX_MARK(1);
 
     // ---- input stage --------------------------------------------------------------------

@@ -30,15 +30,17 @@ int sm_count() {
     return cached[dev];
 }
 
+#ifdef AFX_EXPERIMENT
 int g_force_pw = 0, g_force_s = 0;  // experiment knobs, 0 = automatic
 int g_cluster_margin = -1;          // experiment knob, < 0 = automatic
+#endif
 
 template <int DT, int TMAX>
 static afx_status launch_gemv_t(const GemvListArgs& a, cudaStream_t st) {
     const void* kerns[3] = {reinterpret_cast<const void*>(sparse_gemv_kernel<DT, TMAX, 256>),
                             reinterpret_cast<const void*>(sparse_gemv_kernel<DT, TMAX, 128>),
                             reinterpret_cast<const void*>(sparse_gemv_kernel<DT, TMAX, 64>)};
-    const GemvShapeChoice c = choose_gemv_shape(a.N, kerns, 0, g_force_pw, g_force_s);
+    const GemvShapeChoice c = choose_gemv_shape(a.N, kerns, 0);
     switch (c.pw) {
         case 256: return launch_clustered(sparse_gemv_kernel<DT, TMAX, 256>, c.S, c.tiles, 0, a, st);
         case 128: return launch_clustered(sparse_gemv_kernel<DT, TMAX, 128>, c.S, c.tiles, 0, a, st);
@@ -56,23 +58,35 @@ static afx_status launch_gemv(const GemvListArgs& a, cudaStream_t st) {
 
 }  // namespace afx
 
-// Not part of the ABI: forces tile width / cluster size for kernel experiments (0 = automatic).
+#ifdef AFX_EXPERIMENT
+// Experiment builds only (not part of the ABI): force tile width / cluster size / margin.
 extern "C" void afx_internal_tune_gemv(int pw, int s) {
     afx::g_force_pw = pw;
     afx::g_force_s = s;
 }
 extern "C" void afx_internal_cluster_margin(int margin) { afx::g_cluster_margin = margin; }
+#endif
+
+extern "C" size_t afx_workspace_bytes(int K_max, int N_max, int T_max) {
+    (void)K_max;
+    (void)N_max;
+    (void)T_max;
+    return 0;  // partial sums meet in (distributed) shared memory: no entry point needs scratch
+}
 
 extern "C" afx_status afx_sparse_gemv(const void* Wt, int dtype, int K, int N, int64_t ldw,
                                       const void* x, int T, const int32_t* idx, const int32_t* count,
-                                      const int32_t* slot, float* y, int accumulate, void* stream) {
+                                      const int32_t* slot, float* y, int accumulate, int32_t* dev_status,
+                                      void* stream) {
     using namespace afx;
     if (Wt == nullptr || x == nullptr || idx == nullptr || count == nullptr || y == nullptr)
         return AFX_ERR_INVALID_ARG;
     if (K <= 0 || N <= 0 || T < 1 || T > AFX_MAX_T || ldw < N) return AFX_ERR_INVALID_ARG;
     if (dtype != AFX_F16 && dtype != AFX_BF16) return AFX_ERR_UNSUPPORTED;
     if ((N & 7) != 0 || (ldw & 7) != 0 || !aligned16(Wt) || !aligned16(y) ||
-        (reinterpret_cast<uintptr_t>(x) & 1u) != 0)
+        (reinterpret_cast<uintptr_t>(x) & 1u) != 0 || (reinterpret_cast<uintptr_t>(idx) & 3u) != 0 ||
+        (reinterpret_cast<uintptr_t>(count) & 3u) != 0 || (reinterpret_cast<uintptr_t>(slot) & 3u) != 0 ||
+        (reinterpret_cast<uintptr_t>(dev_status) & 3u) != 0)
         return AFX_ERR_ALIGNMENT;
     if ((N + 63) / 64 > 65535) return AFX_ERR_CAPACITY;
     GemvListArgs a;
@@ -89,6 +103,7 @@ extern "C" afx_status afx_sparse_gemv(const void* Wt, int dtype, int K, int N, i
     a.ep.y = y;
     a.ep.out_bits = nullptr;
     a.ep.N = N;
+    a.status = dev_status;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     return dtype == AFX_F16 ? launch_gemv<AFX_F16>(a, st) : launch_gemv<AFX_BF16>(a, st);
 }

@@ -208,6 +208,7 @@ struct GemvListArgs {
     const int32_t* slot;
     int accumulate;
     EpilogueArgs ep;
+    int32_t* status;  // device status word or NULL
 };
 
 // grid = (S, tiles), cluster = (S, 1, 1).
@@ -220,12 +221,17 @@ __device__ __forceinline__ void gemv_list_block(const GemvListArgs& a, GemvSmem<
     const int S = gridDim.x, s = blockIdx.x, tile = blockIdx.y;
     const int T = a.T;
     cluster_arrive();
-    // Programmatic dependent launch: let the next grid in the stream be scheduled as soon as
-    // SM resources free up, and touch global memory only once the previous grid is complete.
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // Programmatic dependent launch: global memory is touched only once the previous grid is
+    // complete, and the next grid in the stream may be scheduled (as SM resources free up)
+    // only after that -- so whatever a grid reads before its own wait was written at least
+    // two grids earlier and is complete.
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     int cnt = *a.count;
-    cnt = max(0, min(cnt, a.K));
+    if (cnt < 0 || cnt > a.K) {
+        if (tid == 0 && s == 0 && tile == 0) report_status(a.status, AFX_ERR_CAPACITY);
+        cnt = max(0, min(cnt, a.K));
+    }
     const int c_lo = static_cast<int>(static_cast<int64_t>(s) * cnt / S);
     const int c_hi = static_cast<int>(static_cast<int64_t>(s + 1) * cnt / S);
     const int out0 = tile * PW + (lane % LPC) * 8;
@@ -241,11 +247,17 @@ __device__ __forceinline__ void gemv_list_block(const GemvListArgs& a, GemvSmem<
         const int staged = min(CAP, c_hi - c0);
         __syncthreads();
         for (int i = tid; i < staged; i += kGemvThreads) {
+            // An entry outside [0, K), or one whose cache slot is negative (a transient that found
+            // no staging row), takes no part: column 0 with x = 0, and the status word says so.
             const int j = a.idx[c0 + i];
-            sm->col[i] = a.slot != nullptr ? a.slot[c0 + i] : j;
+            const int col = a.slot != nullptr ? a.slot[c0 + i] : j;
+            const bool in_range = static_cast<unsigned>(j) < static_cast<unsigned>(a.K);
+            const bool ok = in_range && col >= 0;
+            if (!ok && tile == 0) report_status(a.status, in_range ? AFX_ERR_CAPACITY : AFX_ERR_INVALID_ARG);
+            sm->col[i] = ok ? col : 0;
 #pragma unroll
             for (int t = 0; t < TMAX; ++t)
-                if (t < T) sm->xv[t][i] = bits_to_float<DT>(a.x[static_cast<size_t>(t) * a.K + j]);
+                if (t < T) sm->xv[t][i] = ok ? bits_to_float<DT>(a.x[static_cast<size_t>(t) * a.K + j]) : 0.0f;
         }
         __syncthreads();
         if (lane_ok) gemv_stream<DT, TMAX, PW, CAP>(a.Wt + out0, a.ldw, T, sm, staged, acc);

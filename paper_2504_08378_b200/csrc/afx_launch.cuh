@@ -86,11 +86,18 @@ struct GemvShapeChoice {
 // Widest tile and largest cluster such that all tiles' clusters are resident at once
 // (one wave) and the block count is as large as possible.  kerns[i] is the kernel
 // instantiated for tile width 256 >> i.
+#ifdef AFX_EXPERIMENT
 extern int g_force_pw, g_force_s;  // experiment knobs (0 = automatic)
 extern int g_cluster_margin;      // experiment knob (< 0 = automatic)
+#endif
 
 inline GemvShapeChoice choose_gemv_shape(int N, const void* const kerns[3], size_t dyn_smem,
-                                         int force_pw = 0, int force_s = 0, int extra_clusters = 0) {
+                                         int extra_clusters = 0) {
+#ifdef AFX_EXPERIMENT
+    const int force_pw = g_force_pw, force_s = g_force_s, force_margin = g_cluster_margin;
+#else
+    constexpr int force_pw = 0, force_s = 0, force_margin = -1;
+#endif
     GemvShapeChoice best = {64, 1, (N + 63) / 64};
     int best_blocks = -1;
     for (int i = 0; i < 3; ++i) {
@@ -103,7 +110,7 @@ inline GemvShapeChoice choose_gemv_shape(int N, const void* const kerns[3], size
             // The occupancy query counts free block slots per GPC; launched behind another
             // kernel, two clusters fewer than it reports were seen resident at once (the
             // last ones then ran as a second wave), so a margin stays free.
-            const int margin = g_cluster_margin >= 0 ? g_cluster_margin : (tiles + 15) / 16 < 2 ? 2 : (tiles + 15) / 16;
+            const int margin = force_margin >= 0 ? force_margin : (tiles + 15) / 16 < 2 ? 2 : (tiles + 15) / 16;
             if (max_active_clusters(kerns[i], S, dyn_smem) >= tiles + extra_clusters + margin) {
                 s_fit = S;
                 break;

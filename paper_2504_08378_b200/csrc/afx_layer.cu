@@ -50,7 +50,7 @@ static afx_status launch_fused_t(const FusedArgs& a, cudaStream_t st) {
     b.side_cluster = (a.idx_out != nullptr || a.count_out != nullptr || a.bitmap_out != nullptr ||
                       a.xnorm_out != nullptr || a.bitmap_pred != nullptr || a.kth_slot != nullptr)
                          ? 1 : 0;
-    const GemvShapeChoice c = choose_gemv_shape(a.N, kerns, dyn, g_force_pw, g_force_s, b.side_cluster);
+    const GemvShapeChoice c = choose_gemv_shape(a.N, kerns, dyn, b.side_cluster);
     if (c.tiles + b.side_cluster > 65535) return AFX_ERR_CAPACITY;
     const int rows = c.tiles + b.side_cluster;
     switch (c.pw) {
@@ -330,14 +330,12 @@ static afx_status check_step(const afx_model* m, int layer, const afx_state* s) 
 
 }  // namespace afx
 
-extern "C" afx_status afx_layer_step(afx_model* m, int layer, afx_state* s, int pos, void* stream) {
-    using namespace afx;
-    afx_status rc = check_step(m, layer, s);
-    if (rc != AFX_OK) return rc;
+namespace afx {
+
+// One of the five kernels of a layer step (which = AFX_STEP_*), on validated arguments.
+static afx_status launch_layer_kernel(afx_model* m, int layer, afx_state* s, int pos, int which, cudaStream_t st) {
     const afx_model_desc& d = m->d;
-    if (pos < 0 || pos >= d.max_seq) return AFX_ERR_INVALID_ARG;
     const afx_layer_desc& L = m->layers[layer];
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
     float* h = reinterpret_cast<float*>(s->blob + s->off_h);
     float* qkv = reinterpret_cast<float*>(s->blob + s->off_qkv);
     uint16_t* attn = reinterpret_cast<uint16_t*>(s->blob + s->off_attn);
@@ -347,69 +345,85 @@ extern "C" afx_status afx_layer_step(afx_model* m, int layer, afx_state* s, int 
     FusedArgs a = {};
     a.T = s->T;
     a.eps = d.rms_eps;
-    // ---- q | k | v ----
-    a.Wt = static_cast<const uint16_t*>(L.w_qkv);
-    a.ldw = m->n_qkv;
-    a.K = d.hidden;
-    a.N = m->n_qkv;
-    a.h = h;
-    a.gain = L.g_attn;
-    a.x = nullptr;
-    a.xnorm_out = reinterpret_cast<uint16_t*>(s->blob + s->off_xnorm[0]);
-    a.ep = {qkv, nullptr, m->n_qkv};
-    plan_selection(m, s, layer, AFX_OP_QKV, true, &a);
-    if ((rc = launch_fused<IN_NORM, EP_STORE>(d.dtype, a, st)) != AFX_OK) return rc;
-    // ---- rotary, cache append, dense attention ----
-    AttnArgs at = {};
-    at.qkv = qkv;
-    at.n_qkv = m->n_qkv;
-    at.q_heads = d.n_heads;
-    at.kv_heads = d.n_kv_heads;
-    at.T = s->T;
-    at.k_cache = static_cast<uint16_t*>(L.k_cache);
-    at.v_cache = static_cast<uint16_t*>(L.v_cache);
-    at.max_seq = d.max_seq;
-    at.pos = pos;
-    at.rope_cos = m->rope;
-    at.rope_sin = m->rope + static_cast<size_t>(d.max_seq) * (kHeadDim / 2);
-    at.out = attn;
-    if ((rc = launch_attention(d.dtype, at, st)) != AFX_OK) return rc;
-    // ---- o ----
-    a.Wt = static_cast<const uint16_t*>(L.w_o);
-    a.ldw = d.hidden;
-    a.K = n_attn;
-    a.N = d.hidden;
-    a.h = nullptr;
-    a.gain = nullptr;
-    a.x = attn;
-    a.xnorm_out = nullptr;
-    a.ep = {h, nullptr, d.hidden};
-    plan_selection(m, s, layer, AFX_OP_O, true, &a);
-    if ((rc = launch_fused<IN_X, EP_ACCUM>(d.dtype, a, st)) != AFX_OK) return rc;
-    // ---- gate | up, silu(gate) * up ----
-    a.Wt = static_cast<const uint16_t*>(L.w_gu);
-    a.ldw = 2 * static_cast<int64_t>(d.mlp);
-    a.K = d.hidden;
-    a.N = 2 * d.mlp;
-    a.h = h;
-    a.gain = L.g_mlp;
-    a.x = nullptr;
-    a.xnorm_out = reinterpret_cast<uint16_t*>(s->blob + s->off_xnorm[1]);
-    a.ep = {nullptr, hm, 2 * d.mlp};
-    plan_selection(m, s, layer, AFX_OP_GU, true, &a);
-    if ((rc = launch_fused<IN_NORM, EP_SILU>(d.dtype, a, st)) != AFX_OK) return rc;
-    // ---- down ----
-    a.Wt = static_cast<const uint16_t*>(L.w_down);
-    a.ldw = d.hidden;
-    a.K = d.mlp;
-    a.N = d.hidden;
-    a.h = nullptr;
-    a.gain = nullptr;
-    a.x = hm;
-    a.xnorm_out = nullptr;
-    a.ep = {h, nullptr, d.hidden};
-    plan_selection(m, s, layer, AFX_OP_DOWN, true, &a);
-    return launch_fused<IN_X, EP_ACCUM>(d.dtype, a, st);
+    switch (which) {
+        case AFX_STEP_QKV:  // q | k | v
+            a.Wt = static_cast<const uint16_t*>(L.w_qkv);
+            a.ldw = m->n_qkv;
+            a.K = d.hidden;
+            a.N = m->n_qkv;
+            a.h = h;
+            a.gain = L.g_attn;
+            a.xnorm_out = reinterpret_cast<uint16_t*>(s->blob + s->off_xnorm[0]);
+            a.ep = {qkv, nullptr, m->n_qkv};
+            plan_selection(m, s, layer, AFX_OP_QKV, true, &a);
+            return launch_fused<IN_NORM, EP_STORE>(d.dtype, a, st);
+        case AFX_STEP_ATTN: {  // rotary, cache append, dense attention
+            AttnArgs at = {};
+            at.qkv = qkv;
+            at.n_qkv = m->n_qkv;
+            at.q_heads = d.n_heads;
+            at.kv_heads = d.n_kv_heads;
+            at.T = s->T;
+            at.k_cache = static_cast<uint16_t*>(L.k_cache);
+            at.v_cache = static_cast<uint16_t*>(L.v_cache);
+            at.max_seq = d.max_seq;
+            at.pos = pos;
+            at.rope_cos = m->rope;
+            at.rope_sin = m->rope + static_cast<size_t>(d.max_seq) * (kHeadDim / 2);
+            at.out = attn;
+            return launch_attention(d.dtype, at, st);
+        }
+        case AFX_STEP_O:
+            a.Wt = static_cast<const uint16_t*>(L.w_o);
+            a.ldw = d.hidden;
+            a.K = n_attn;
+            a.N = d.hidden;
+            a.x = attn;
+            a.ep = {h, nullptr, d.hidden};
+            plan_selection(m, s, layer, AFX_OP_O, true, &a);
+            return launch_fused<IN_X, EP_ACCUM>(d.dtype, a, st);
+        case AFX_STEP_GU:  // gate | up, silu(gate) * up
+            a.Wt = static_cast<const uint16_t*>(L.w_gu);
+            a.ldw = 2 * static_cast<int64_t>(d.mlp);
+            a.K = d.hidden;
+            a.N = 2 * d.mlp;
+            a.h = h;
+            a.gain = L.g_mlp;
+            a.xnorm_out = reinterpret_cast<uint16_t*>(s->blob + s->off_xnorm[1]);
+            a.ep = {nullptr, hm, 2 * d.mlp};
+            plan_selection(m, s, layer, AFX_OP_GU, true, &a);
+            return launch_fused<IN_NORM, EP_SILU>(d.dtype, a, st);
+        case AFX_STEP_DOWN:
+            a.Wt = static_cast<const uint16_t*>(L.w_down);
+            a.ldw = d.hidden;
+            a.K = d.mlp;
+            a.N = d.hidden;
+            a.x = hm;
+            a.ep = {h, nullptr, d.hidden};
+            plan_selection(m, s, layer, AFX_OP_DOWN, true, &a);
+            return launch_fused<IN_X, EP_ACCUM>(d.dtype, a, st);
+        default: return AFX_ERR_INVALID_ARG;
+    }
+}
+
+}  // namespace afx
+
+extern "C" afx_status afx_layer_step(afx_model* m, int layer, afx_state* s, int pos, void* stream) {
+    using namespace afx;
+    afx_status rc = check_step(m, layer, s);
+    if (rc != AFX_OK) return rc;
+    if (pos < 0 || pos >= m->d.max_seq) return AFX_ERR_INVALID_ARG;
+    for (int which = AFX_STEP_QKV; which <= AFX_STEP_DOWN; ++which)
+        if ((rc = launch_layer_kernel(m, layer, s, pos, which, static_cast<cudaStream_t>(stream))) != AFX_OK) return rc;
+    return AFX_OK;
+}
+
+extern "C" afx_status afx_layer_kernel(afx_model* m, int layer, afx_state* s, int pos, int which, void* stream) {
+    using namespace afx;
+    afx_status rc = check_step(m, layer, s);
+    if (rc != AFX_OK) return rc;
+    if (pos < 0 || pos >= m->d.max_seq || which < AFX_STEP_QKV || which > AFX_STEP_DOWN) return AFX_ERR_INVALID_ARG;
+    return launch_layer_kernel(m, layer, s, pos, which, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" afx_status afx_mlp_block(afx_model* m, int layer, afx_state* s, const void* x, float* y,
@@ -492,16 +506,27 @@ static __device__ __align__(256) uint16_t g_noalloc_hm[AFX_MAX_T * kNoAllocMaxMl
 
 // Device address of g_noalloc_hm on the current device (host code only sees a stand-in for
 // the symbol; the address has to be asked for, once per device, with that device current).
-static afx_status noalloc_scratch(uint16_t** out) {
+// The address is cached for the life of the process: it does not survive cudaDeviceReset.
+// The lookup must not run while `st` is capturing (it is not a stream operation and may
+// initialise the module on the device), so a first call under capture is refused.
+static afx_status noalloc_scratch(cudaStream_t st, uint16_t** out) {
+    constexpr int kMaxDevices = 64;
     static std::mutex mu;
-    static uint16_t* addr[64] = {};
+    static uint16_t* addr[kMaxDevices] = {};
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) {
         cudaGetLastError();
         return AFX_ERR_CUDA;
     }
+    if (dev >= kMaxDevices) return AFX_ERR_CAPACITY;
     std::lock_guard<std::mutex> lock(mu);
     if (addr[dev] == nullptr) {
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) {
+            cudaGetLastError();
+            return AFX_ERR_CUDA;
+        }
+        if (cap != cudaStreamCaptureStatusNone) return AFX_ERR_INVALID_ARG;
         void* p = nullptr;
         if (cudaGetSymbolAddress(&p, g_noalloc_hm) != cudaSuccess || p == nullptr) {
             cudaGetLastError();
@@ -529,10 +554,10 @@ extern "C" afx_status afx_mlp_block_noalloc(const void* w_gu, const void* w_down
     if ((hidden & 7) != 0 || (mlp & 7) != 0 || !aligned16(w_gu) || !aligned16(w_down) || !aligned16(y) ||
         (reinterpret_cast<uintptr_t>(x) & 1u) != 0)
         return AFX_ERR_ALIGNMENT;
-    uint16_t* hm = nullptr;
-    afx_status rc = noalloc_scratch(&hm);
-    if (rc != AFX_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint16_t* hm = nullptr;
+    afx_status rc = noalloc_scratch(st, &hm);
+    if (rc != AFX_OK) return rc;
     // Nothing in hm has to start from zero: the first kernel writes all T * mlp values that
     // the second one reads.
     FusedArgs a = {};
@@ -558,7 +583,8 @@ extern "C" afx_status afx_mlp_block_noalloc(const void* w_gu, const void* w_down
     return launch_fused<IN_X, EP_STORE>(dtype, a, st);
 }
 
-// Not part of the ABI: clusters of S blocks of the bf16 one-token operator (tile width pw,
+#ifdef AFX_EXPERIMENT
+// Experiment builds only (not part of the ABI): clusters of S blocks of the bf16 one-token operator (tile width pw,
 // plain input of K channels, h += epilogue) that the occupancy query reports as co-resident.
 extern "C" int afx_internal_max_clusters(int pw, int S, int K) {
     using namespace afx;
@@ -568,3 +594,4 @@ extern "C" int afx_internal_max_clusters(int pw, int S, int K) {
                                  : reinterpret_cast<const void*>(fused_op_kernel<AFX_BF16, 1, 64, IN_X, EP_ACCUM>);
     return max_active_clusters(kern, S, dyn);
 }
+#endif

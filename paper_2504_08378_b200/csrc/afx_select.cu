@@ -67,39 +67,46 @@ select_kernel(const uint16_t* __restrict__ x, int K, int T, int mode, int k, flo
 }
 
 // miss = A \ P (ascending), hit = |A & P|.  One block; each warp owns a contiguous run of
-// list positions so that the output keeps A's order.
+// list positions so that the output keeps A's order.  An entry outside [0, K) is neither a
+// hit nor a miss; the status word reports it.
 __global__ void __launch_bounds__(kSelectThreads, 1)
 diff_kernel(const int32_t* __restrict__ idxA, const int32_t* __restrict__ cntA,
             const uint32_t* __restrict__ bitmapP, int K, int32_t* __restrict__ miss,
-            int32_t* __restrict__ miss_count, int32_t* __restrict__ hit_count) {
-    __shared__ int scan[33];
+            int32_t* __restrict__ miss_count, int32_t* __restrict__ hit_count, int32_t* __restrict__ status) {
+    __shared__ int scan[2][33];
     int n = *cntA;
-    n = max(0, min(n, K));
+    if (n < 0 || n > K) {
+        if (threadIdx.x == 0) report_status(status, AFX_ERR_CAPACITY);
+        n = max(0, min(n, K));
+    }
     const int lane = lane_id();
     const uint32_t lt_mask = (1u << lane) - 1u;
     const int nchunks = (n + 31) >> 5;
     const int nw = blockDim.x >> 5;
     const int per = (nchunks + nw - 1) / nw;
     const int c0 = min(nchunks, warp_id() * per), c1 = min(nchunks, c0 + per);
-    int cm = 0;
+    int cm = 0, cbad = 0;
     for (int c = c0; c < c1; ++c) {
         const int p = (c << 5) + lane;
-        bool m = false;
+        bool m = false, bad = false;
         if (p < n) {
             const int j = idxA[p];
-            m = ((bitmapP[j >> 5] >> (j & 31)) & 1u) == 0u;
+            bad = static_cast<unsigned>(j) >= static_cast<unsigned>(K);
+            m = !bad && ((bitmapP[j >> 5] >> (j & 31)) & 1u) == 0u;
         }
         cm += __popc(__ballot_sync(0xFFFFFFFFu, m));
+        cbad += __popc(__ballot_sync(0xFFFFFFFFu, bad));
     }
-    int total;
-    int base = warp_prefix(cm, scan, total);
+    int total, total_bad;
+    int base = warp_prefix(cm, scan[0], total);
+    warp_prefix(cbad, scan[1], total_bad);
     for (int c = c0; c < c1; ++c) {
         const int p = (c << 5) + lane;
         bool m = false;
         int j = 0;
         if (p < n) {
             j = idxA[p];
-            m = ((bitmapP[j >> 5] >> (j & 31)) & 1u) == 0u;
+            m = static_cast<unsigned>(j) < static_cast<unsigned>(K) && ((bitmapP[j >> 5] >> (j & 31)) & 1u) == 0u;
         }
         const uint32_t b = __ballot_sync(0xFFFFFFFFu, m);
         if (m) miss[base + __popc(b & lt_mask)] = j;
@@ -107,7 +114,8 @@ diff_kernel(const int32_t* __restrict__ idxA, const int32_t* __restrict__ cntA,
     }
     if (threadIdx.x == 0) {
         *miss_count = total;
-        *hit_count = n - total;
+        *hit_count = n - total - total_bad;
+        if (total_bad > 0) report_status(status, AFX_ERR_INVALID_ARG);
     }
 }
 
@@ -139,13 +147,19 @@ extern "C" afx_status afx_select_active(const void* x, int dtype, int K, int T, 
 
 extern "C" afx_status afx_diff_active(const int32_t* idxA, const int32_t* cntA,
                                       const uint32_t* bitmapP, int K, int32_t* miss,
-                                      int32_t* miss_count, int32_t* hit_count, void* stream) {
+                                      int32_t* miss_count, int32_t* hit_count, int32_t* dev_status,
+                                      void* stream) {
     using namespace afx;
     if (idxA == nullptr || cntA == nullptr || bitmapP == nullptr || miss == nullptr ||
         miss_count == nullptr || hit_count == nullptr)
         return AFX_ERR_INVALID_ARG;
     if (K <= 0 || K > (1 << 20)) return AFX_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(idxA) & 3u) || (reinterpret_cast<uintptr_t>(cntA) & 3u) ||
+        (reinterpret_cast<uintptr_t>(bitmapP) & 3u) || (reinterpret_cast<uintptr_t>(miss) & 3u) ||
+        (reinterpret_cast<uintptr_t>(miss_count) & 3u) || (reinterpret_cast<uintptr_t>(hit_count) & 3u) ||
+        (reinterpret_cast<uintptr_t>(dev_status) & 3u))
+        return AFX_ERR_ALIGNMENT;
     diff_kernel<<<1, kSelectThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-        idxA, cntA, bitmapP, K, miss, miss_count, hit_count);
+        idxA, cntA, bitmapP, K, miss, miss_count, hit_count, dev_status);
     return launch_status();
 }

@@ -121,6 +121,9 @@ class DecoderModel:
     def layer_step(self, layer: int, pos: int, stream=None):
         afx.afx_layer_step(self.handle, layer, self.state, pos, stream)
 
+    def layer_kernel(self, layer: int, pos: int, which: int, stream=None):
+        afx.afx_layer_kernel(self.handle, layer, self.state, pos, which, stream)
+
     def decode_step(self, pos: int, stream=None):
         for layer in range(self.n_layers):
             afx.afx_layer_step(self.handle, layer, self.state, pos, stream)

@@ -3,6 +3,7 @@ arguments on the host before anything is launched."""
 import ctypes
 import os
 import re
+import subprocess
 
 import pytest
 
@@ -27,6 +28,18 @@ def test_every_declared_symbol_is_exported():
     assert "afx_select_active" in declared and "afx_sparse_gemv" in declared
     for name in declared:
         assert hasattr(L, name), f"{name} declared in include/ but not exported"
+
+
+def test_no_exported_afx_symbol_is_undeclared():
+    """The shipped library exports exactly the afx_* functions the header declares: no
+    experiment knobs, no tracing hooks (dynamic symbol table read with nm, nothing else)."""
+    out = subprocess.check_output(["nm", "-D", "--defined-only", afx.lib()._name], text=True)
+    exported = {ln.split()[-1] for ln in out.splitlines() if ln.split() and ln.split()[-1].startswith("afx_")}
+    assert exported == set(_declared_symbols()), exported ^ set(_declared_symbols())
+
+
+def test_no_entry_point_needs_scratch_memory():
+    assert afx.afx_workspace_bytes(32768, 1 << 20, 8) == 0 and afx.afx_workspace_bytes(1, 8, 1) == 0
 
 
 def test_binding_has_the_same_names():
@@ -84,8 +97,13 @@ def test_gemv_rejects_bad_arguments_on_the_host():
     assert call(ldw=36) == 2                       # ldw not a multiple of 8
     assert call(Wt=FAKE + 8) == 2 and call(y=FAKE + 4) == 2
     assert call(N=8 * 600000, ldw=8 * 600000) == 3  # more column tiles than a grid holds
+    assert call(idx=FAKE + 2) == 2 and call(slot=FAKE + 1) == 2
+    with pytest.raises(afx.AfxError) as e:
+        afx.afx_sparse_gemv(FAKE, 1, 64, 32, 32, FAKE, 1, FAKE, FAKE, None, FAKE, 0, stream=0, dev_status=FAKE + 2)
+    assert e.value.status == 2
 
 
 def test_diff_rejects_bad_arguments_on_the_host():
     assert _status(afx.afx_diff_active, None, FAKE, FAKE, 8, FAKE, FAKE, FAKE) == 1
     assert _status(afx.afx_diff_active, FAKE, FAKE, FAKE, 0, FAKE, FAKE, FAKE) == 1
+    assert _status(afx.afx_diff_active, FAKE + 2, FAKE, FAKE, 8, FAKE, FAKE, FAKE) == 2

@@ -9,7 +9,7 @@ import oracle
 import oracle.layer as ol
 from paper_2504_08378_b200 import afx, synth
 from gpu_util import dev_i32, rel_err
-from test_gpu_layer import OPN, TOL, bits_np, check_layer_stages, make, oracle_weights, ulp_close
+from test_gpu_layer import OPN, TOL, bits_np, check_layer_stages, hm_close, make, oracle_weights
 
 pytestmark = pytest.mark.gpu
 
@@ -49,7 +49,7 @@ def test_config2_mlp_block_7b_threshold_sweep():
         if p:
             assert abs(stats[2][0] / hidden - (1 - p / 100)) < 0.03  # realised sparsity near the target
         hm_gpu = bits_np(m.bits(afx.BUF_HM))
-        assert ulp_close(hm_gpu, ref["hm"], frac_exact=0.97, dt=dt), p
+        assert hm_close(host, dt, mlp, x, ref["idx_gu"], hm_gpu, ref["hm"]), p
         idx_d = m.idx(afx.OP_DOWN).cpu().numpy()[: stats[3][0]]
         assert np.array_equal(idx_d, oracle.select_active(hm_gpu, dt, oracle.THRESHOLD, tau=tau_d))
         y_ref = oracle.sparse_gemv(host["w_down"], dt, hidden, hm_gpu, idx_d)

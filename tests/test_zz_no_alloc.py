@@ -14,6 +14,8 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
+import oracle.layer as ol
 from paper_2504_08378_b200 import afx, synth
 from paper_2504_08378_b200.model import DecoderModel
 from gpu_util import rel_err
@@ -48,6 +50,35 @@ def test_noalloc_mlp_block_matches_mlp_block_twice(dt, T, mode):
         assert np.isfinite(ref).all()
         assert rel_err(y.cpu().numpy(), ref) <= TOL, f"call {call}"
     m.close()
+
+
+@pytest.mark.parametrize("dt", ["bf16", "f16"])
+def test_noalloc_two_calls_enqueued_back_to_back_match_the_oracle(dt):
+    """Two calls with different inputs on one stream, nothing in between: the second call's
+    first kernel rewrites the shared array that the first call's second kernel reads, so the
+    stream order between them is all that keeps them apart.  Both results against the CPU
+    oracle's MLP block (which also pins the result itself, not only the scratch plumbing)."""
+    hidden, mlp, T = 1024, 2752, 1
+    L = synth.layer_weights(78, 0, hidden, 8, 8, mlp, dt)
+    kk = [0, 0, hidden // 2, mlp // 2]
+    w_gu = _dev(synth.interleave_gate_up(L["w_gate"], L["w_up"]))
+    w_down = _dev(L["w_down"])
+    xs = [synth.laplace_bits(78, 30 + c, (T, hidden), dt) for c in range(2)]
+    xd = [_dev(x) for x in xs]
+    ys = [torch.full((T, hidden), float("nan"), device="cuda") for _ in range(2)]
+    torch.cuda.synchronize()
+    for c in range(2):
+        afx.afx_mlp_block_noalloc(w_gu, w_down, dt, hidden, mlp, xd[c], T, afx.MODE_TOPK, kk[2], 0.0, kk[3], 0.0, ys[c])
+    torch.cuda.synchronize()
+    cfg = ol.Config(dt, hidden, 8, 8, mlp, mode=oracle.TOPK)
+    lw = ol.LayerWeights(None, None, L["w_gate"], L["w_up"], L["w_down"], None, None, k={"gu": kk[2], "down": kk[3]})
+    for c in range(2):
+        ref = ol.mlp_block(cfg, lw, xs[c])
+        # The intermediate silu(gate)*up stays inside the library, so this comparison cannot be
+        # teacher-forced at the second operator: both sides round the intermediate to 16 bits
+        # from sums that differ in their last fp32 bits, a few percent of its elements come out
+        # one step apart (2^-8 relative for bf16), and that carries about 1e-3 into y.
+        assert rel_err(ys[c].cpu().numpy(), ref["y"]) <= 5e-3, c
 
 
 def test_noalloc_rejects_sizes_beyond_the_fixed_array():
