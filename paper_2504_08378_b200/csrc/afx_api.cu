@@ -22,8 +22,8 @@ extern "C" const char* afx_status_string(afx_status s) {
 
 #ifdef AFX_TRACE
 #include <cuda_runtime.h>
-__device__ long long afx_trace_buf[5 * 512 * 16];
+__device__ long long afx_trace_buf[8 * 512 * 16];
 extern "C" int afx_trace_read(long long* host_out) {
-    return cudaMemcpyFromSymbol(host_out, afx_trace_buf, sizeof(long long) * 5 * 512 * 16) == cudaSuccess ? 0 : 1;
+    return cudaMemcpyFromSymbol(host_out, afx_trace_buf, sizeof(long long) * 8 * 512 * 16) == cudaSuccess ? 0 : 1;
 }
 #endif

@@ -80,6 +80,7 @@ __device__ __forceinline__ void attention_block(const AttnArgs& a, AttnSmem* sm)
     const float qscale = rsqrtf(static_cast<float>(kHeadDim)) * 1.4426950408889634f;
     const uint32_t half_mask = 0xFFFFu << (16 * half);  // the two halves of a warp work on different keys
 
+    AFX_TRACE_REGION(0);
     AFX_MARK(0);
     uint16_t* kc = a.k_cache + static_cast<size_t>(t) * a.max_seq * a.kv_heads * kHeadDim;
     uint16_t* vc = a.v_cache + static_cast<size_t>(t) * a.max_seq * a.kv_heads * kHeadDim;

@@ -15,6 +15,9 @@
 #define AFX_MARK(i) \
     do {            \
     } while (0)
+#define AFX_TRACE_REGION(r) \
+    do {                    \
+    } while (0)
 #endif
 
 namespace afx {
@@ -49,6 +52,39 @@ __device__ __forceinline__ void unpack8(const uint4& raw, float (&w)[8]) {
         } else {
             w[2 * i] = __uint_as_float(r[i] << 16);
             w[2 * i + 1] = __uint_as_float(r[i] & 0xFFFF0000u);
+        }
+    }
+}
+
+// ---- packed fp32 pairs (two-wide fused multiply-add of sm_100) ------------------------
+
+typedef unsigned long long f32x2;  // two fp32 values in one 64-bit register pair (low, high)
+
+__device__ __forceinline__ f32x2 pack_f32x2(float lo, float hi) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(f32x2 v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+// acc = a * b + acc on both halves, each exactly as a scalar fma.rn.f32.
+__device__ __forceinline__ void fma_f32x2(f32x2& acc, f32x2 a, f32x2 b) {
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(a), "l"(b));
+}
+
+// Eight packed 16-bit weights (one 128-bit load) as four fp32 pairs (weights 2i, 2i+1).
+template <int DT>
+__device__ __forceinline__ void unpack8_pairs(const uint4& raw, f32x2 (&w)[4]) {
+    const uint32_t r[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        if (DT == AFX_F16) {
+            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&r[i]));
+            w[i] = pack_f32x2(f.x, f.y);
+        } else {
+            const uint32_t lo = r[i] << 16, hi = r[i] & 0xFFFF0000u;
+            asm("mov.b64 %0, {%1, %2};" : "=l"(w[i]) : "r"(lo), "r"(hi));
         }
     }
 }

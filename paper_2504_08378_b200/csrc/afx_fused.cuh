@@ -82,8 +82,11 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
     GemvSmem<TMAX, CAP>* sm = reinterpret_cast<GemvSmem<TMAX, CAP>*>(work);
     float* red16 = reinterpret_cast<float*>(sel->hist);  // block reduction of the norm
 
+    const uint32_t ld16 = static_cast<uint32_t>(a.ldw >> 3);  // row stride in 16-byte units (the launcher checked the range)
     const bool own = (a.idx_in == nullptr);
     const bool topk = own && a.mode == AFX_MODE_TOPK && a.k > 0 && a.k < K;
+    // kernel kinds of a decode step: 1 q|k|v, 2 gate|up, 3 down (the wider plain input), 4 o
+    AFX_TRACE_REGION(IN == IN_NORM ? (EP == EP_SILU ? 2 : 1) : (K > a.N ? 3 : 4));
     AFX_MARK(0);
     if (!side) cluster_arrive();  // the side cluster never meets
     if (topk) block_clear_key_hist<kGemvThreads>(hist);  // does not depend on the previous kernel
@@ -219,7 +222,7 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
                     xt, K, a.mode, a.k, a.tau, hist, t == 0, sel, true, pos0, cnt, [&](int j, int pos, uint16_t bits) {
                         const int p = pos - e_lo;
                         if (p >= 0 && p < e_n) {  // the histogram is dead by now: its memory is the staging area
-                            sm->col[p] = j;
+                            sm->col[p] = static_cast<uint32_t>(j) * ld16;
                             sm->xv[0][p] = bits_to_float<DT>(bits);
                         }
                     }, e_lo, e_lo + e_n, hint, xchg);
@@ -286,7 +289,7 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
                     for_each_owned_active(fl, K, pos0, [&](int j, int pos) {
                         const int p = pos - c0;
                         if (p >= 0 && p < staged) {
-                            sm->col[p] = j;
+                            sm->col[p] = static_cast<uint32_t>(j) * ld16;
 #pragma unroll
                             for (int t = 0; t < TMAX; ++t)
                                 if (t < T) sm->xv[t][p] = bits_to_float<DT>(x_at(t, j));
@@ -296,7 +299,7 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
             } else {
                 for (int i = tid; i < staged; i += kGemvThreads) {
                     const int j = a.idx_in[c0 + i];
-                    sm->col[i] = j;
+                    sm->col[i] = static_cast<uint32_t>(j) * ld16;
 #pragma unroll
                     for (int t = 0; t < TMAX; ++t)
                         if (t < T) sm->xv[t][i] = bits_to_float<DT>(x_at(t, j));
@@ -305,7 +308,8 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
         }
         __syncthreads();
         AFX_MARK(4);
-        if (lane_ok) gemv_stream<DT, TMAX, PW, CAP>(a.Wt + out0, a.ldw, T, sm, staged, acc);
+        if (lane_ok)
+            gemv_stream<DT, TMAX, PW, CAP, false>(reinterpret_cast<const uint4*>(a.Wt + out0), T, sm, staged, acc);
     }
     AFX_MARK(5);
 

@@ -25,9 +25,12 @@ constexpr int kGemvUnroll = 8;
 constexpr int kMaxCluster = 8;
 
 // Shared memory of one block.  CAP = channels whose (column, x) pairs are staged at once.
+// A column is staged as its offset from the start of the weights in 16-byte units
+// (row * ldw / 8: 32 bits cover operators of up to 64 GB), so that a load address is one
+// multiply-add away.
 template <int TMAX, int CAP>
 struct GemvSmem {
-    int col[CAP];
+    uint32_t col[CAP];
     float xv[TMAX][CAP];
     __align__(16) float red[kGemvWarps][256];  // per-warp sums of one token
 };
@@ -60,9 +63,14 @@ struct EpilogueArgs {
     int N;               // outputs of the operator (columns of Wt)
 };
 
-// Streams the staged channels [0, staged) of one tile: acc[t][q] += xv[t][p] * W[col[p]][out0+q].
-template <int DT, int TMAX, int PW, int CAP>
-__device__ __forceinline__ void gemv_stream(const uint16_t* __restrict__ wbase, int64_t ldw, int T,
+// Streams the staged channels [0, staged) of one tile: acc[t][q] += xv[t][p] * W[row(p)][out0+q].
+// wbase16 points at this lane's 8 outputs of row 0; sm->col[p] is row(p)'s offset in 16-byte
+// units.  Products and sums are two-wide fused multiply-adds (bitwise the scalar fma.rn
+// results).  SPLIT: full batches of U loads per lane run without per-load guards and a guarded
+// batch finishes (fewer instructions; the extra loop costs registers, which the fused operator
+// kernels with their selection state do not have to spare).
+template <int DT, int TMAX, int PW, int CAP, bool SPLIT>
+__device__ __forceinline__ void gemv_stream(const uint4* __restrict__ wbase16, int T,
                                             const GemvSmem<TMAX, CAP>* sm, int staged,
                                             float (&acc)[TMAX][8]) {
     constexpr int LPC = PW / 8;             // lanes per channel piece
@@ -71,30 +79,45 @@ __device__ __forceinline__ void gemv_stream(const uint16_t* __restrict__ wbase, 
     constexpr int U = kGemvUnroll;
     const int lane = threadIdx.x & 31;
     const int eg = (threadIdx.x >> 5) * SUB + lane / LPC;
-    for (int p = eg; p < staged; p += EG * U) {
-        uint4 raw[U];
+    f32x2 a2[TMAX][4];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int pp = p + u * EG;
-            if (pp < staged) raw[u] = ld_stream_16B(wbase + static_cast<int64_t>(sm->col[pp]) * ldw);
-        }
+    for (int t = 0; t < TMAX; ++t)
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int pp = p + u * EG;
-            if (pp < staged) {
-                float w[8];
-                unpack8<DT>(raw[u], w);
+        for (int i = 0; i < 4; ++i) a2[t][i] = pack_f32x2(acc[t][2 * i], acc[t][2 * i + 1]);
+    auto consume = [&](const uint4& raw, int pp) {
+        f32x2 w[4];
+        unpack8_pairs<DT>(raw, w);
 #pragma unroll
-                for (int t = 0; t < TMAX; ++t) {
-                    if (t < T) {
-                        const float xv = sm->xv[t][pp];
+        for (int t = 0; t < TMAX; ++t) {
+            if (t < T) {
+                const float xv = sm->xv[t][pp];
+                const f32x2 x2 = pack_f32x2(xv, xv);
 #pragma unroll
-                        for (int q = 0; q < 8; ++q) acc[t][q] = fmaf(xv, w[q], acc[t][q]);
-                    }
-                }
+                for (int i = 0; i < 4; ++i) fma_f32x2(a2[t][i], w[i], x2);
             }
         }
+    };
+    // one batch: U loads per lane in flight, then their products
+    auto batch = [&](int p, bool guarded) {
+        uint4 raw[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (!guarded || p + u * EG < staged) raw[u] = ld_stream_16B(wbase16 + sm->col[p + u * EG]);
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (!guarded || p + u * EG < staged) consume(raw[u], p + u * EG);
+    };
+    if (SPLIT) {
+        int p = eg;
+        for (; p + (U - 1) * EG < staged; p += EG * U) batch(p, false);
+        if (p < staged) batch(p, true);
+    } else {
+        for (int p = eg; p < staged; p += EG * U) batch(p, true);
     }
+#pragma unroll
+    for (int t = 0; t < TMAX; ++t)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) unpack_f32x2(a2[t][i], acc[t][2 * i], acc[t][2 * i + 1]);
 }
 
 // Block-level then cluster-level meeting of the sums of one tile, then the epilogue:
@@ -236,6 +259,8 @@ __device__ __forceinline__ void gemv_list_block(const GemvListArgs& a, GemvSmem<
     const int c_hi = static_cast<int>(static_cast<int64_t>(s + 1) * cnt / S);
     const int out0 = tile * PW + (lane % LPC) * 8;
     const bool lane_ok = out0 < a.N;
+    const uint64_t ld16 = static_cast<uint64_t>(a.ldw >> 3);  // row stride in 16-byte units
+    const uint4* wbase16 = reinterpret_cast<const uint4*>(a.Wt + out0);
 
     float acc[TMAX][8];
 #pragma unroll
@@ -252,15 +277,16 @@ __device__ __forceinline__ void gemv_list_block(const GemvListArgs& a, GemvSmem<
             const int j = a.idx[c0 + i];
             const int col = a.slot != nullptr ? a.slot[c0 + i] : j;
             const bool in_range = static_cast<unsigned>(j) < static_cast<unsigned>(a.K);
-            const bool ok = in_range && col >= 0;
+            const uint64_t off = static_cast<uint64_t>(col < 0 ? 0 : col) * ld16;
+            const bool ok = in_range && col >= 0 && off + static_cast<uint64_t>(a.N >> 3) <= 0x100000000ull;
             if (!ok && tile == 0) report_status(a.status, in_range ? AFX_ERR_CAPACITY : AFX_ERR_INVALID_ARG);
-            sm->col[i] = ok ? col : 0;
+            sm->col[i] = ok ? static_cast<uint32_t>(off) : 0u;
 #pragma unroll
             for (int t = 0; t < TMAX; ++t)
                 if (t < T) sm->xv[t][i] = ok ? bits_to_float<DT>(a.x[static_cast<size_t>(t) * a.K + j]) : 0.0f;
         }
         __syncthreads();
-        if (lane_ok) gemv_stream<DT, TMAX, PW, CAP>(a.Wt + out0, a.ldw, T, sm, staged, acc);
+        if (lane_ok) gemv_stream<DT, TMAX, PW, CAP, true>(wbase16, T, sm, staged, acc);
     }
     if (a.accumulate)
         gemv_finish_tile<DT, TMAX, PW, CAP, EP_ACCUM>(acc, T, tile, sm, recv, a.ep);

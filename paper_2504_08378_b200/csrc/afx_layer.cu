@@ -41,6 +41,8 @@ static cudaError_t launch_attention_rep(const cudaLaunchConfig_t& cfg, int rep, 
 
 template <int DT, int TMAX, int IN, int EP>
 static afx_status launch_fused_t(const FusedArgs& a, cudaStream_t st) {
+    // staged column offsets are 32-bit counts of 16-byte units
+    if (static_cast<uint64_t>(a.K) * static_cast<uint64_t>(a.ldw >> 3) > 0x100000000ull) return AFX_ERR_CAPACITY;
     const size_t dyn = fused_dyn_smem(IN, a.K, a.T);
     const void* kerns[3] = {reinterpret_cast<const void*>(fused_op_kernel<DT, TMAX, 256, IN, EP>),
                             reinterpret_cast<const void*>(fused_op_kernel<DT, TMAX, 128, IN, EP>),

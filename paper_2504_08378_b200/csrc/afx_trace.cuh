@@ -1,17 +1,26 @@
-// Recording form of AFX_MARK, used only by timing-study builds (-DAFX_TRACE): thread 0 of
-// every block stores the SM clock of mark i (0..14) into afx_trace_buf, in one of five
-// regions told apart by the launch shape (256-thread blocks; 5-, 3- and other cluster widths,
-// the last split by dynamic shared memory above / below 80 KB); slots 15 and 14 of a block
-// hold the global nanosecond timer and the SM id at its mark 0.
+// Recording form of the stage marks, used only by timing-study builds (-DAFX_TRACE).
+// AFX_TRACE_REGION(r) (thread 0, at kernel start) names the kernel kind, 0..7; AFX_MARK(i)
+// then stores the SM clock of mark i (0..13) of that block into afx_trace_buf
+// [region][block % 512][16]; slots 15 and 14 hold the global nanosecond timer and the SM id
+// at mark 0.
 #pragma once
 
 extern __device__ long long afx_trace_buf[];
+
+__device__ __forceinline__ int* afx_trace_region_ptr() {
+    __shared__ int region;
+    return &region;
+}
+
+#define AFX_TRACE_REGION(r)                                   \
+    do {                                                      \
+        if (threadIdx.x == 0) *afx_trace_region_ptr() = (r);  \
+    } while (0)
+
 #define AFX_MARK(i)                                                                                   \
     do {                                                                                              \
         if (threadIdx.x == 0) {                                                                       \
-            unsigned dyn_;                                                                            \
-            asm volatile("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn_));                            \
-            const int region_ = blockDim.x == 256 ? 0 : (gridDim.x == 5 ? 1 : (gridDim.x == 3 ? 2 : (dyn_ > 80000u ? 3 : 4))); \
+            const int region_ = *afx_trace_region_ptr();                                              \
             long long* slot_ = afx_trace_buf + (region_ * 512 + (blockIdx.y * gridDim.x + blockIdx.x) % 512) * 16; \
             slot_[(i)] = clock64();                                                                   \
             if ((i) == 0) {                                                                           \
