@@ -213,3 +213,54 @@ class LfuCache:
 
     def cached(self) -> np.ndarray:
         return np.sort(self.chan_of[self.chan_of >= 0])
+
+
+# ---- cross-layer-group preloading (Sec. 3 "Data layout", Sec. 4 operations PL and L) ----
+
+def group_layout_offset(layer: int, channel: int, n_layers: int, d: int, K: int, ldw: int) -> int:
+    """Element offset of (layer, channel) of ONE operator type in the reordered host image
+    (Sec. 3 "Data layout", Fig. "reordered weights in a 4-layers group"): groups in layer order;
+    inside a group the order is channel id, then layer id:
+    [Ch0_L, Ch0_L+1, .., Ch0_L+d-1, Ch1_L, ..].  A group of dg layers (dg = d except for a
+    shorter last group) therefore stores channel j as one run of dg columns."""
+    g, i = layer // d, layer % d
+    dg = min(d, n_layers - g * d)
+    return ((g * d * K) + channel * dg + i) * ldw   # all earlier groups are full: g*d layers * K columns
+
+
+def pack_group_layout(per_layer, d: int) -> np.ndarray:
+    """per_layer: list of [K][ldw] uint16 arrays (one operator type, layer order) -> the host
+    image in the layout of group_layout_offset, written with plain loops over its definition."""
+    L = len(per_layer)
+    K, ldw = per_layer[0].shape
+    out = np.empty(L * K * ldw, np.uint16)
+    for l in range(L):
+        for j in range(K):
+            o = group_layout_offset(l, j, L, d, K, ldw)
+            out[o:o + ldw] = per_layer[l][j]
+    return out
+
+
+def swap_acquire(P, A, rows_pred: int, rows_miss: int):
+    """Where each active channel of a layer is found after the preload of its group (Sec. 3:
+    what the prediction covered was preloaded, "the missed active weights during preloading will
+    be on-demand loaded"): the c-th predicted channel sits in row c (c < rows_pred; predicted
+    channels beyond rows_pred were not preloaded); a channel of A that was not preloaded is
+    loaded on demand into row rows_pred + m, m = its rank among this layer's on-demand loads,
+    or gets -1 when rows_miss is exhausted.  Returns dict(slot, ondemand, hits, overflow)."""
+    P = [int(j) for j in P][:rows_pred]
+    row_of = {j: c for c, j in enumerate(P)}
+    slot, ondemand, overflow = [], [], 0
+    for j in (int(v) for v in A):
+        if j in row_of:
+            slot.append(row_of[j])
+        else:
+            m = len(ondemand) + overflow
+            if m < rows_miss:
+                slot.append(rows_pred + m)
+                ondemand.append(j)
+            else:
+                slot.append(-1)
+                overflow += 1
+    return dict(slot=np.array(slot, np.int32), ondemand=np.array(ondemand, np.int32),
+                hits=len(slot) - len(ondemand) - overflow, overflow=overflow)
