@@ -345,6 +345,93 @@ afx_status afx_cache_fetch(afx_cache* cache, const int32_t* idx, const int32_t* 
  * cached), usage[K].  Synchronises the stream. */
 afx_status afx_cache_snapshot(afx_cache* cache, int32_t* host_slot_of, uint32_t* host_usage, void* stream);
 
+/* ------------------------------------------------------------------------------------------
+ * Cross-layer-group weight swapping (Sec. 3 "Cross-layer Active Weight Preloading" with its
+ * data layout, and the PL "preload" / L "on-demand load" operations of the pipeline of Sec. 4).
+ * One object serves ONE operator type (say W_down) of all layers.  Its weights live in pinned
+ * HOST memory in the paper's reordered layout: groups of `group` consecutive layers (group g =
+ * layers g*group .. g*group+group-1, the last one possibly shorter); inside a group the columns
+ * are ordered by channel id, then layer id -- [Ch0_L, Ch0_L+1, .., Ch1_L, Ch1_L+1, ..] -- so
+ * the columns one predicted channel needs in all layers of the group are ONE contiguous chunk.
+ *
+ * While the layers of a group are computed, afx_swap_preload copies the chunks of the channels
+ * PREDICTED for the next group (the active list of an earlier layer's activation) into device
+ * rows on a loader stream; when a layer's actual activation is known, afx_swap_acquire maps
+ * every active channel to its preloaded row or loads it on demand (one column, this layer
+ * only) and returns the slot list that afx_sparse_gemv takes.  Stream events stand in for the
+ * paper's request / complete signals between the loading and the computing thread; no kernel
+ * spins on a flag.
+ * ------------------------------------------------------------------------------------------ */
+
+typedef struct afx_swap afx_swap; /* opaque, HOST object owning small DEVICE tables, two pairs of events and
+                                     (unless one is given) a loader stream */
+
+typedef struct {
+    int32_t dtype;        /* AFX_F16 / AFX_BF16                                                  */
+    int32_t n_layers;     /* layers that have this operator                                      */
+    int32_t group;        /* d: layers per cross-layer group (>= 1)                              */
+    int32_t K, N;         /* channels of the operator, values per channel (N % 8 == 0)           */
+    int64_t ldw;          /* row stride in elements of the host image AND the device rows        */
+    int32_t rows_pred;    /* device rows per layer for preloaded channels (a longer prediction   */
+                          /* is cut: its first rows_pred channels are preloaded)                 */
+    int32_t rows_miss;    /* device rows per layer for on-demand channels                        */
+    const void* host_base;/* HOST, page-locked, n_layers * K rows of ldw in the group layout     */
+    void* dev_rows;       /* DEVICE, afx_swap_device_bytes() bytes, 16-byte aligned:             */
+                          /* [2 buffers][group][rows_pred + rows_miss][ldw]; groups alternate    */
+    void* loader_stream;  /* cudaStream_t the preloads run on, or NULL: the object creates one   */
+} afx_swap_desc;
+
+typedef struct {
+    int32_t hits;      /* active channels found preloaded                                        */
+    int32_t ondemand;  /* active channels loaded on demand by this acquire                       */
+    int32_t overflow;  /* active channels that found no on-demand row (slot -1)                  */
+    int32_t preloaded; /* channels the group's preload brought in                                */
+    uint64_t bytes_preload;  /* host -> device bytes of that preload (preloaded * layers * N * 2) */
+    uint64_t bytes_ondemand; /* host -> device bytes of this acquire (ondemand * N * 2)          */
+} afx_swap_stats;
+
+/* Element offset of column (layer, channel) in the host image (HOST arithmetic, no GPU needed);
+ * (size_t)-1 for arguments out of range. */
+size_t afx_swap_host_offset(int n_layers, int group, int K, int64_t ldw, int layer, int channel);
+
+/* Re-orders per-layer operator tensors (HOST pointers per_layer[l] -> [K][ldw] 16-bit values)
+ * into the group layout at host_out (n_layers * K * ldw values).  Plain host copies. */
+afx_status afx_swap_pack_host(const void* const* per_layer, int n_layers, int group, int K, int64_t ldw,
+                              void* host_out);
+
+/* Bytes of dev_rows the descriptor needs (0 for a bad descriptor). */
+size_t afx_swap_device_bytes(const afx_swap_desc* desc);
+
+/* Resolves the device view of host_base (AFX_ERR_INVALID_ARG when it is not page-locked),
+ * allocates the tables (cudaMalloc, about 12 bytes per channel), creates the events and, if
+ * none was given, the loader stream.  afx_swap_destroy releases them. */
+afx_status afx_swap_create(const afx_swap_desc* desc, afx_swap** out);
+afx_status afx_swap_destroy(afx_swap* swap);
+
+/*
+ * PL: preload group `group_index` from the predicted list idxP[0 .. *cntP) (DEVICE, ascending, as
+ * afx_select_active or a layer step writes it).  Enqueued on the loader stream behind everything
+ * enqueued on compute_stream so far (the list must have been produced there); predicted
+ * channel c goes to row c of every layer of the group.  copy_blocks: thread blocks of the copy
+ * kernel (0 = 32; it reads host memory over PCIe and needs few).  Call it only after the
+ * compute stream has been given all work of group_index - 2, whose buffer it overwrites.
+ */
+afx_status afx_swap_preload(afx_swap* swap, int group_index, const int32_t* idxP, const int32_t* cntP,
+                            int copy_blocks, int32_t* dev_status, void* compute_stream);
+
+/*
+ * L: the layer's actual active list idxA[0 .. *cntA) is known.  On compute_stream: waits for the
+ * preload of the layer's group (if one was requested; otherwise nothing counts as preloaded),
+ * writes slot_out[c] = row of idxA[c] (preloaded row, or rows_pred + m for the m-th on-demand
+ * channel, or -1 when the on-demand rows are used up: AFX_ERR_CAPACITY in dev_status, and
+ * afx_sparse_gemv leaves such channels out), copies the on-demand columns, fills *stats
+ * (DEVICE or NULL).  *rows_out (HOST) receives the DEVICE address of this layer's rows: pass it
+ * as Wt, with slot_out as slot, to afx_sparse_gemv on the same stream.
+ */
+afx_status afx_swap_acquire(afx_swap* swap, int layer, const int32_t* idxA, const int32_t* cntA,
+                            int32_t* slot_out, afx_swap_stats* stats, int32_t* dev_status, void* compute_stream,
+                            const void** rows_out);
+
 /*
  * The MLP block without any allocation (the paper has no counterpart: this entry point exists
  * for the integration, not for the method).  Same result as afx_mlp_block on the same weights

@@ -54,6 +54,19 @@ class CacheStats(ctypes.Structure):
                 ("bytes_fetched", ctypes.c_uint64)]
 
 
+class SwapDesc(ctypes.Structure):
+    """afx_swap_desc"""
+    _fields_ = [("dtype", c_int32), ("n_layers", c_int32), ("group", c_int32), ("K", c_int32), ("N", c_int32),
+                ("ldw", c_int64), ("rows_pred", c_int32), ("rows_miss", c_int32), ("host_base", c_void_p),
+                ("dev_rows", c_void_p), ("loader_stream", c_void_p)]
+
+
+class SwapStats(ctypes.Structure):
+    """afx_swap_stats"""
+    _fields_ = [("hits", c_int32), ("ondemand", c_int32), ("overflow", c_int32), ("preloaded", c_int32),
+                ("bytes_preload", ctypes.c_uint64), ("bytes_ondemand", ctypes.c_uint64)]
+
+
 class AfxError(RuntimeError):
     def __init__(self, fn: str, status: int):
         self.status = status
@@ -101,6 +114,16 @@ def lib() -> ctypes.CDLL:
         L.afx_cache_install.argtypes = [c_void_p, c_void_p, c_int, c_void_p]
         L.afx_cache_fetch.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
         L.afx_cache_snapshot.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p]
+        L.afx_swap_host_offset.restype = c_size_t
+        L.afx_swap_host_offset.argtypes = [c_int, c_int, c_int, c_int64, c_int, c_int]
+        L.afx_swap_pack_host.argtypes = [ctypes.POINTER(c_void_p), c_int, c_int, c_int, c_int64, c_void_p]
+        L.afx_swap_device_bytes.restype = c_size_t
+        L.afx_swap_device_bytes.argtypes = [ctypes.POINTER(SwapDesc)]
+        L.afx_swap_create.argtypes = [ctypes.POINTER(SwapDesc), ctypes.POINTER(c_void_p)]
+        L.afx_swap_destroy.argtypes = [c_void_p]
+        L.afx_swap_preload.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_int, c_void_p, c_void_p]
+        L.afx_swap_acquire.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                       ctypes.POINTER(c_void_p)]
         L.afx_mlp_block_noalloc.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_void_p, c_int, c_int, c_int,
                                             c_float, c_int, c_float, c_void_p, c_void_p]
         _lib = L
@@ -267,3 +290,44 @@ def afx_cache_snapshot(cache: int, K: int, stream=None):
     _check("afx_cache_snapshot",
            lib().afx_cache_snapshot(cache, slot_of.ctypes.data, usage.ctypes.data, _stream(stream)))
     return slot_of, usage
+
+
+def afx_swap_host_offset(n_layers: int, group: int, K: int, ldw: int, layer: int, channel: int) -> int:
+    """Element offset of (layer, channel) in the cross-layer-group host image (host arithmetic)."""
+    v = int(lib().afx_swap_host_offset(int(n_layers), int(group), int(K), int(ldw), int(layer), int(channel)))
+    if v == (1 << 64) - 1:
+        raise AfxError("afx_swap_host_offset", 1)
+    return v
+
+
+def afx_swap_pack_host(per_layer_ptrs, n_layers: int, group: int, K: int, ldw: int, host_out):
+    """per_layer_ptrs: host addresses of the per-layer [K][ldw] tensors; host_out: host address."""
+    arr = (c_void_p * n_layers)(*[int(p) for p in per_layer_ptrs])
+    _check("afx_swap_pack_host", lib().afx_swap_pack_host(arr, int(n_layers), int(group), int(K), int(ldw), host_out))
+
+
+def afx_swap_device_bytes(desc: SwapDesc) -> int:
+    return int(lib().afx_swap_device_bytes(ctypes.byref(desc)))
+
+
+def afx_swap_create(desc: SwapDesc) -> int:
+    out = c_void_p(0)
+    _check("afx_swap_create", lib().afx_swap_create(ctypes.byref(desc), ctypes.byref(out)))
+    return out.value
+
+
+def afx_swap_destroy(swap: int):
+    _check("afx_swap_destroy", lib().afx_swap_destroy(swap))
+
+
+def afx_swap_preload(swap: int, group_index: int, idxP, cntP, copy_blocks: int = 0, stream=None, dev_status=None):
+    _check("afx_swap_preload", lib().afx_swap_preload(swap, int(group_index), _ptr(idxP), _ptr(cntP), int(copy_blocks),
+                                                      _ptr(dev_status), _stream(stream)))
+
+
+def afx_swap_acquire(swap: int, layer: int, idxA, cntA, slot_out, stats=None, stream=None, dev_status=None) -> int:
+    """Returns the device address of the layer's rows (the Wt argument of afx_sparse_gemv)."""
+    rows = c_void_p(0)
+    _check("afx_swap_acquire", lib().afx_swap_acquire(swap, int(layer), _ptr(idxA), _ptr(cntA), _ptr(slot_out),
+                                                      _ptr(stats), _ptr(dev_status), _stream(stream), ctypes.byref(rows)))
+    return rows.value

@@ -221,6 +221,8 @@ __device__ __forceinline__ void gemv_finish_tile(float (&acc)[TMAX][8], int T, i
     }
 }
 
+constexpr uint32_t kSkippedEntry = 0xFFFFFFFFu;  // staged column of a list entry that takes no part
+
 struct GemvListArgs {
     const uint16_t* Wt;
     int64_t ldw;
@@ -268,24 +270,46 @@ __device__ __forceinline__ void gemv_list_block(const GemvListArgs& a, GemvSmem<
 #pragma unroll
         for (int q = 0; q < 8; ++q) acc[t][q] = 0.0f;
 
+    __shared__ int first_ok;
     for (int c0 = c_lo; c0 < c_hi; c0 += CAP) {
-        const int staged = min(CAP, c_hi - c0);
+        int staged = min(CAP, c_hi - c0);
         __syncthreads();
+        bool skipped = false;
         for (int i = tid; i < staged; i += kGemvThreads) {
-            // An entry outside [0, K), or one whose cache slot is negative (a transient that found
-            // no staging row), takes no part: column 0 with x = 0, and the status word says so.
+            // An entry outside [0, K), or one whose cache slot is negative (a channel that found
+            // no row), takes no part: x = 0, and the status word says so.
             const int j = a.idx[c0 + i];
             const int col = a.slot != nullptr ? a.slot[c0 + i] : j;
             const bool in_range = static_cast<unsigned>(j) < static_cast<unsigned>(a.K);
             const uint64_t off = static_cast<uint64_t>(col < 0 ? 0 : col) * ld16;
-            const bool ok = in_range && col >= 0 && off + static_cast<uint64_t>(a.N >> 3) <= 0x100000000ull;
+            const bool ok = in_range && col >= 0 && off + static_cast<uint64_t>(a.N >> 3) <= 0xFFFFFFFFull;
             if (!ok && tile == 0) report_status(a.status, in_range ? AFX_ERR_CAPACITY : AFX_ERR_INVALID_ARG);
-            sm->col[i] = ok ? static_cast<uint32_t>(off) : 0u;
+            skipped |= !ok;
+            sm->col[i] = ok ? static_cast<uint32_t>(off) : kSkippedEntry;
 #pragma unroll
             for (int t = 0; t < TMAX; ++t)
                 if (t < T) sm->xv[t][i] = ok ? bits_to_float<DT>(a.x[static_cast<size_t>(t) * a.K + j]) : 0.0f;
         }
-        __syncthreads();
+        if (__syncthreads_or(skipped)) {
+            // Rare.  A skipped entry still costs a load in the streaming loop; whatever it reads
+            // is multiplied by 0, so it must read weights (finite), not a row nobody filled:
+            // send it to the column of the first entry that does take part.
+            if (tid == 0) first_ok = staged;
+            __syncthreads();
+            for (int i = tid; i < staged; i += kGemvThreads)
+                if (sm->col[i] != kSkippedEntry) atomicMin(&first_ok, i);
+            __syncthreads();
+            const int f = first_ok;
+            if (f < staged) {
+                const uint32_t safe = sm->col[f];
+                __syncthreads();
+                for (int i = tid; i < staged; i += kGemvThreads)
+                    if (sm->col[i] == kSkippedEntry) sm->col[i] = safe;
+            } else {
+                staged = 0;  // nothing in this part of the list takes part
+            }
+            __syncthreads();
+        }
         if (lane_ok) gemv_stream<DT, TMAX, PW, CAP, true>(wbase16, T, sm, staged, acc);
     }
     if (a.accumulate)
