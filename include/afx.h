@@ -432,6 +432,81 @@ afx_status afx_swap_acquire(afx_swap* swap, int layer, const int32_t* idxA, cons
                             int32_t* slot_out, afx_swap_stats* stats, int32_t* dev_status, void* compute_stream,
                             const void** rows_out);
 
+/* ------------------------------------------------------------------------------------------
+ * Cost model of the swapping pipeline and the greedy parameter search (Sec. 4.1 "Elastic and
+ * Optimized LLM Execution", Eq. 1-9 and the symbol table).  HOST arithmetic; sizes in bytes,
+ * bandwidths in bytes per second, times in seconds.
+ * ------------------------------------------------------------------------------------------ */
+
+typedef struct {
+    double sp;             /* sparsity of the model                                            */
+    double hr;             /* average hit rate of the weight cache                             */
+    double si;             /* average similarity inside a cross-layer group                    */
+    int32_t N;             /* layers per cross-layer group                                     */
+    int32_t n_layers;      /* layers of the model (0: T_token counts two groups)               */
+    double S_l;            /* size of one layer                                                */
+    double bw_mem;         /* BW_mem                                                           */
+    double bw_flash_small; /* BW_flash^small: single-channel reads (on-demand loads)           */
+    double bw_flash_large; /* BW_flash^large: group-chunk reads (preloads)                     */
+    double M_cache, M_kv;  /* memory of the weight cache and of the KV cache                   */
+} afx_cost_params;
+
+typedef struct {
+    double M_cl;      /* Eq. 9: S_l (1 - sp) N                                                  */
+    double M;         /* Eq. 8: M_cl + M_cache + M_kv                                           */
+    double T_load;    /* Eq. 3: M_cl (1 - hr) / BW_flash^small                                  */
+    double T_comp;    /* Eq. 4: M_cl / BW_mem                                                   */
+    double T_onload;  /* Eq. 6: S_l (1 - sp)(1 - hr)(1 - si) / BW_flash^small                   */
+    double T_preload; /* Eq. 7: M_cl (1 - hr) / BW_flash^large                                  */
+    double T_overlap; /* Eq. 5: T_onload + max(T_preload, T_comp)                               */
+    double T_decode;  /* Eq. 1 as printed: T_load + T_overlap + T_comp                          */
+    double T_token;   /* the same with one overlap stage per further group of the model:        */
+                      /* T_load + (ceil(n_layers / N) - 1) T_overlap + T_comp                   */
+} afx_cost;
+
+afx_status afx_cost_eval(const afx_cost_params* params, afx_cost* out);
+
+/* Why the search stopped growing the group. */
+#define AFX_COST_STOP_BALANCED 0 /* T_preload <= T_comp: preloading hides behind computation   */
+#define AFX_COST_STOP_GAIN 1     /* one more layer lowered T_preload per layer by < min_gain   */
+#define AFX_COST_STOP_MEMORY 2   /* a larger group no longer fits M_max                        */
+#define AFX_COST_STOP_N_MAX 3    /* N_max (or the layer count) reached                         */
+
+typedef struct {
+    double S_m, S_l;             /* size of the model, of one layer                             */
+    int32_t n_layers;
+    double M_max, M_kv;          /* memory budget; fixed KV-cache memory                        */
+    double bw_mem, bw_flash_small;
+    int32_t n_chunk;             /* measured large-read bandwidth by chunk size (HOST arrays,   */
+    const double* chunk_bytes;   /* chunk_bytes ascending); a group of N layers reads chunks of */
+    const double* chunk_bw;      /* N * column_bytes                                            */
+    double column_bytes;         /* bytes of one channel of one layer's operator                */
+    int32_t n_hr;                /* measured cache hit rate by cache size as a fraction of S_m  */
+    const double* hr_cache_frac; /* (HOST arrays, ascending)                                    */
+    const double* hr_value;
+    double si;                   /* cross-layer similarity                                      */
+    double min_gain;             /* relative drop of T_preload per layer that still pays        */
+    int32_t N_max;
+} afx_cost_search_in;
+
+typedef struct {
+    double sp;        /* 1 - M_max / S_m (not below 0)                                          */
+    int32_t N;        /* chosen layers per group                                                */
+    double M_cache;   /* what the budget leaves for the weight cache                            */
+    double hr;        /* hit rate read from the table at that cache size                        */
+    double bw_flash_large;
+    afx_cost cost;
+    int32_t stop_reason;
+} afx_cost_choice;
+
+/*
+ * The paper's greedy search: sparsity from the memory budget, then the group grows one layer
+ * at a time (larger chunks read faster) until preloading is no slower than computing, the
+ * gain per added layer falls below min_gain, or the budget is exhausted; the memory a group
+ * does not need goes to the weight cache.  AFX_ERR_CAPACITY when even one layer does not fit.
+ */
+afx_status afx_cost_search(const afx_cost_search_in* in, afx_cost_choice* out);
+
 /*
  * The MLP block without any allocation (the paper has no counterpart: this entry point exists
  * for the integration, not for the method).  Same result as afx_mlp_block on the same weights

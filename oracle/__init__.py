@@ -264,3 +264,27 @@ def swap_acquire(P, A, rows_pred: int, rows_miss: int):
                 overflow += 1
     return dict(slot=np.array(slot, np.int32), ondemand=np.array(ondemand, np.int32),
                 hits=len(slot) - len(ondemand) - overflow, overflow=overflow)
+
+
+# ---- cost model of the swapping pipeline (Sec. 4.1, Eq. 1-9) ----
+
+def cost_model(sp, hr, si, N, S_l, bw_mem, bw_flash_small, bw_flash_large, M_cache=0.0, M_kv=0.0, n_layers=None):
+    """Eq. 1-9 written out one by one, in the paper's symbols (sizes in bytes, bandwidths in
+    bytes/s, times in s).  T_decode is Eq. 1 as printed: the first group's load, ONE overlap
+    stage and the last group's computation.  With n_layers given, T_token also counts one
+    overlap stage per further group (n_layers / N groups: first load, groups - 1 overlap
+    stages, last computation)."""
+    M_cl = S_l * (1.0 - sp) * N                                            # Eq. 9
+    M = M_cl + M_cache + M_kv                                              # Eq. 8
+    T_load = M_cl * (1.0 - hr) / bw_flash_small                            # Eq. 3
+    T_comp = M_cl / bw_mem                                                 # Eq. 4
+    T_onload = S_l * (1.0 - sp) * (1.0 - hr) * (1.0 - si) / bw_flash_small  # Eq. 6
+    T_preload = M_cl * (1.0 - hr) / bw_flash_large                         # Eq. 7
+    T_overlap = T_onload + max(T_preload, T_comp)                          # Eq. 5
+    T_decode = T_load + T_overlap + T_comp                                 # Eq. 1
+    out = dict(M_cl=M_cl, M=M, T_load=T_load, T_comp=T_comp, T_onload=T_onload, T_preload=T_preload,
+               T_overlap=T_overlap, T_decode=T_decode)
+    if n_layers is not None:
+        groups = -(-n_layers // N)
+        out["T_token"] = T_load + (groups - 1) * T_overlap + T_comp
+    return out

@@ -67,6 +67,39 @@ class SwapStats(ctypes.Structure):
                 ("bytes_preload", ctypes.c_uint64), ("bytes_ondemand", ctypes.c_uint64)]
 
 
+class CostParams(ctypes.Structure):
+    """afx_cost_params"""
+    _fields_ = [("sp", ctypes.c_double), ("hr", ctypes.c_double), ("si", ctypes.c_double), ("N", c_int32),
+                ("n_layers", c_int32), ("S_l", ctypes.c_double), ("bw_mem", ctypes.c_double),
+                ("bw_flash_small", ctypes.c_double), ("bw_flash_large", ctypes.c_double), ("M_cache", ctypes.c_double),
+                ("M_kv", ctypes.c_double)]
+
+
+class Cost(ctypes.Structure):
+    """afx_cost"""
+    _fields_ = [(n, ctypes.c_double) for n in ("M_cl", "M", "T_load", "T_comp", "T_onload", "T_preload", "T_overlap",
+                                               "T_decode", "T_token")]
+
+    def as_dict(self):
+        return {n: getattr(self, n) for n, _ in self._fields_}
+
+
+class CostSearchIn(ctypes.Structure):
+    """afx_cost_search_in"""
+    _fields_ = [("S_m", ctypes.c_double), ("S_l", ctypes.c_double), ("n_layers", c_int32), ("M_max", ctypes.c_double),
+                ("M_kv", ctypes.c_double), ("bw_mem", ctypes.c_double), ("bw_flash_small", ctypes.c_double),
+                ("n_chunk", c_int32), ("chunk_bytes", ctypes.POINTER(ctypes.c_double)),
+                ("chunk_bw", ctypes.POINTER(ctypes.c_double)), ("column_bytes", ctypes.c_double), ("n_hr", c_int32),
+                ("hr_cache_frac", ctypes.POINTER(ctypes.c_double)), ("hr_value", ctypes.POINTER(ctypes.c_double)),
+                ("si", ctypes.c_double), ("min_gain", ctypes.c_double), ("N_max", c_int32)]
+
+
+class CostChoice(ctypes.Structure):
+    """afx_cost_choice"""
+    _fields_ = [("sp", ctypes.c_double), ("N", c_int32), ("M_cache", ctypes.c_double), ("hr", ctypes.c_double),
+                ("bw_flash_large", ctypes.c_double), ("cost", Cost), ("stop_reason", c_int32)]
+
+
 class AfxError(RuntimeError):
     def __init__(self, fn: str, status: int):
         self.status = status
@@ -124,6 +157,8 @@ def lib() -> ctypes.CDLL:
         L.afx_swap_preload.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_int, c_void_p, c_void_p]
         L.afx_swap_acquire.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                        ctypes.POINTER(c_void_p)]
+        L.afx_cost_eval.argtypes = [ctypes.POINTER(CostParams), ctypes.POINTER(Cost)]
+        L.afx_cost_search.argtypes = [ctypes.POINTER(CostSearchIn), ctypes.POINTER(CostChoice)]
         L.afx_mlp_block_noalloc.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_void_p, c_int, c_int, c_int,
                                             c_float, c_int, c_float, c_void_p, c_void_p]
         _lib = L
@@ -331,3 +366,25 @@ def afx_swap_acquire(swap: int, layer: int, idxA, cntA, slot_out, stats=None, st
     _check("afx_swap_acquire", lib().afx_swap_acquire(swap, int(layer), _ptr(idxA), _ptr(cntA), _ptr(slot_out),
                                                       _ptr(stats), _ptr(dev_status), _stream(stream), ctypes.byref(rows)))
     return rows.value
+
+
+def afx_cost_eval(**kw) -> dict:
+    """Eq. 1-9 for the given afx_cost_params fields; returns the afx_cost fields as a dict."""
+    out = Cost()
+    _check("afx_cost_eval", lib().afx_cost_eval(ctypes.byref(CostParams(**kw)), ctypes.byref(out)))
+    return out.as_dict()
+
+
+def afx_cost_search(chunk_table, hr_table, **kw) -> dict:
+    """chunk_table: [(chunk bytes, bytes/s)], hr_table: [(cache size / S_m, hit rate)], both
+    ascending; the other afx_cost_search_in fields by keyword."""
+    cb = (ctypes.c_double * len(chunk_table))(*[float(a) for a, _ in chunk_table])
+    cw = (ctypes.c_double * len(chunk_table))(*[float(b) for _, b in chunk_table])
+    hf = (ctypes.c_double * len(hr_table))(*[float(a) for a, _ in hr_table])
+    hv = (ctypes.c_double * len(hr_table))(*[float(b) for _, b in hr_table])
+    arg = CostSearchIn(n_chunk=len(chunk_table), chunk_bytes=cb, chunk_bw=cw, n_hr=len(hr_table), hr_cache_frac=hf,
+                       hr_value=hv, **kw)
+    out = CostChoice()
+    _check("afx_cost_search", lib().afx_cost_search(ctypes.byref(arg), ctypes.byref(out)))
+    return dict(sp=out.sp, N=out.N, M_cache=out.M_cache, hr=out.hr, bw_flash_large=out.bw_flash_large,
+                stop_reason=out.stop_reason, cost=out.cost.as_dict())
