@@ -134,3 +134,35 @@ def decoder_layer(cfg: Config, lw: LayerWeights, h, kc, vc, pos: int, layer: int
                 xl.pred[op] = rec["newpred_" + op]
     rec.update(xnorm_qkv=xa, qkv=qkv, attn=attn, h1=h1, xnorm_gu=xm, hm=hm, h=h2)
     return rec
+
+
+# ---- mixture-of-experts MLP (the Mixtral-shaped deployment of Sec. 1 / Sec. 7.2) ----
+
+def moe_router(x_bits, w_router, dtype: str, top: int = 2):
+    """Dense router of a sparse mixture-of-experts layer for ONE token: logits = W_r x over all
+    channels (the router stays dense, only the experts' operators are sparse), the `top`
+    experts by logit (equal logits: the lower expert id first), their weights the softmax over
+    the chosen logits.  w_router: [hidden][E] bit patterns, channel-contiguous.
+    Returns (expert ids in rank order, weights, logits)."""
+    x = oracle.decode(np.asarray(x_bits, np.uint16).reshape(-1), dtype)
+    W = oracle.decode(w_router, dtype)
+    logits = np.zeros(W.shape[1])
+    for j in range(W.shape[0]):          # ascending channel order, fp64
+        logits += x[j] * W[j]
+    order = sorted(range(W.shape[1]), key=lambda e: (-logits[e], e))[:top]
+    z = np.exp(logits[order] - logits[order[0]])
+    return np.array(order, np.int32), z / z.sum(), logits
+
+
+def moe_block(cfg: Config, x_bits, w_router, experts, top: int = 2):
+    """y = sum over the chosen experts of weight * W_down_e(silu(W_gate_e x) * W_up_e x), every
+    expert operator on the active channels of its own input (mlp_block); experts: list of
+    LayerWeights (only gate / up / down and their k / tau are used); one token."""
+    ids, w, logits = moe_router(x_bits, w_router, cfg.dtype, top)
+    y = np.zeros((1, cfg.hidden))
+    parts = []
+    for e, we in zip(ids, w):
+        part = mlp_block(cfg, experts[int(e)], x_bits)
+        parts.append(part)
+        y = y + we * part["y"]
+    return dict(experts=ids, weights=w, logits=logits, parts=parts, y=y)
