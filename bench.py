@@ -476,6 +476,8 @@ def run_afx(args):
         variants["config4_llama13b_step"] = variant_config4(st)
         variants["config5_llama70b_host_weights_cache"] = cache70b_measure(2, 64, st)
         variants["config5_cross_layer_group_preload"] = swap70b_measure(4, 3, groups=(0, 2), st=st)
+        variants["cost_model"] = cost_model_report(peak, variants["config5_cross_layer_group_preload"],
+                                                   variants["config5_llama70b_host_weights_cache"])
     clocks = sampler.stop()
 
     if rank == 0:
@@ -981,6 +983,28 @@ def swap70b_measure(n_layers, tokens, groups=(0, 1, 2, 4), st=None, lead="first"
             "speedup_over_serial": {kk: round(base / v["ms_per_token"], 3) for kk, v in results.items()} if base else None,
             "paper_context": "the paper reports 4.1x at 4 layers per group over serial loading on phone flash, where small "
                              "reads are far slower than large ones (Sec. 7.3)"}
+
+
+def cost_model_report(hbm_gbs, swap, cache):
+    """The paper's cost model (Eq. 1-9) and greedy search fed with what this run measured: HBM
+    bandwidth, host-link throughput of single-column reads (no preloading) and of group chunks
+    (preloading with d layers per group), the cache hit rate at a 30 % cache; for a 70B-shaped
+    8-layer stack (13.7 GB) under a budget of half its size."""
+    from paper_2504_08378_b200 import afx
+    S_l = 1711276032.0
+    groups = swap["groups"]
+    small = groups["group0"]["pcie_gbs"] * 1e9
+    column = 16384.0  # one channel of a 8192-wide operator
+    chunk = sorted((int(kk[5:]) * column, v["pcie_gbs"] * 1e9) for kk, v in groups.items() if kk != "group0")
+    hr = [(0.0, 0.0), (0.3, cache["value"])]
+    pick = afx.afx_cost_search(chunk, hr, S_m=8 * S_l, S_l=S_l, n_layers=8, M_max=4 * S_l, M_kv=8 * 2 * 2049 * 8 * 128 * 2.0,
+                               bw_mem=hbm_gbs * 1e9, bw_flash_small=small, column_bytes=column, si=0.8, min_gain=0.05,
+                               N_max=4)
+    return {"inputs": {"bw_mem_gbs": hbm_gbs, "bw_link_small_gbs": round(small / 1e9, 1),
+                       "bw_link_by_chunk_gbs": [(int(a), round(b / 1e9, 1)) for a, b in chunk], "hit_rate_at_30pct_cache": cache["value"]},
+            "choice": {"sp": round(pick["sp"], 4), "layers_per_group": pick["N"], "M_cache_bytes": int(pick["M_cache"]),
+                       "hr": round(pick["hr"], 4), "stop_reason": ["balanced", "gain", "memory", "n_max"][pick["stop_reason"]]},
+            "predicted_ms": {kk: round(v * 1e3, 3) for kk, v in pick["cost"].items() if kk.startswith("T_")}}
 
 
 def run_swap70b(args):
