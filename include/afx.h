@@ -507,6 +507,48 @@ typedef struct {
  */
 afx_status afx_cost_search(const afx_cost_search_in* in, afx_cost_choice* out);
 
+/* ------------------------------------------------------------------------------------------
+ * Mixture-of-experts MLP block for one token (the Mixtral-8x7B deployment of Sec. 1 and the
+ * evaluation; the paper applies the same active-weight selection inside every expert).  The
+ * router stays dense; each chosen expert's gate|up and down operators run on the active
+ * channels of their own input, as in afx_mlp_block:
+ *
+ *     logits = W_r x;  e_1..e_top = the experts of largest logit (ties: lower id first);
+ *     p = softmax(logits[e_1..e_top]);  y (+)= sum_r p_r * W_down[e_r](silu(W_gate[e_r] x) * W_up[e_r] x)
+ *
+ * The experts are chosen ON THE DEVICE (no host round trip): the kernels take their weights
+ * from DEVICE tables of device pointers, indexed by what the router kernel wrote.  1 + 2*top
+ * kernels on `stream`.
+ * ------------------------------------------------------------------------------------------ */
+
+typedef struct {
+    int32_t dtype;        /* AFX_F16 / AFX_BF16                                                  */
+    int32_t hidden, mlp;  /* model width, expert MLP width (multiples of 8, <= 32768)            */
+    int32_t n_experts;    /* 1 .. 16                                                             */
+    int32_t top;          /* experts per token, 1 .. min(4, n_experts)                           */
+    int32_t select_mode;  /* AFX_MODE_*: selection inside the experts                            */
+    int32_t k_gu, k_down; /* top-k counts of the two expert operators                            */
+    float tau_gu, tau_down;
+    const void* w_router; /* DEVICE [hidden][ld_router] 16-bit, channel-contiguous, first        */
+    int64_t ld_router;    /* n_experts values of a row used (ld_router >= n_experts)             */
+    const void* w_gu_table;   /* DEVICE array of n_experts DEVICE pointers: [hidden][2*mlp], the  */
+                              /* interleaved gate|up layout of afx_layer_desc, 16-byte aligned   */
+    const void* w_down_table; /* DEVICE array of n_experts DEVICE pointers: [mlp][hidden]         */
+} afx_moe_desc;
+
+/* Bytes of DEVICE workspace afx_moe_block needs (256-byte aligned): router results and the
+ * chosen experts' intermediate vectors.  0 for a bad descriptor. */
+size_t afx_moe_workspace_bytes(const afx_moe_desc* desc);
+
+/*
+ *   x   DEVICE [hidden] 16-bit (already normalised);  y DEVICE [hidden] fp32, 16-byte aligned;
+ *   accumulate = 0 overwrites y, 1 adds to it (the residual stream).
+ * After the call the workspace starts with float logits[16], int32 experts[4], float
+ * weights[4] (for inspection).
+ */
+afx_status afx_moe_block(const afx_moe_desc* desc, const void* x, float* y, int accumulate, void* workspace,
+                         size_t workspace_bytes, void* stream);
+
 /*
  * The MLP block without any allocation (the paper has no counterpart: this entry point exists
  * for the integration, not for the method).  Same result as afx_mlp_block on the same weights

@@ -100,6 +100,14 @@ class CostChoice(ctypes.Structure):
                 ("bw_flash_large", ctypes.c_double), ("cost", Cost), ("stop_reason", c_int32)]
 
 
+class MoeDesc(ctypes.Structure):
+    """afx_moe_desc"""
+    _fields_ = [("dtype", c_int32), ("hidden", c_int32), ("mlp", c_int32), ("n_experts", c_int32), ("top", c_int32),
+                ("select_mode", c_int32), ("k_gu", c_int32), ("k_down", c_int32), ("tau_gu", c_float),
+                ("tau_down", c_float), ("w_router", c_void_p), ("ld_router", c_int64), ("w_gu_table", c_void_p),
+                ("w_down_table", c_void_p)]
+
+
 class AfxError(RuntimeError):
     def __init__(self, fn: str, status: int):
         self.status = status
@@ -159,6 +167,9 @@ def lib() -> ctypes.CDLL:
                                        ctypes.POINTER(c_void_p)]
         L.afx_cost_eval.argtypes = [ctypes.POINTER(CostParams), ctypes.POINTER(Cost)]
         L.afx_cost_search.argtypes = [ctypes.POINTER(CostSearchIn), ctypes.POINTER(CostChoice)]
+        L.afx_moe_workspace_bytes.restype = c_size_t
+        L.afx_moe_workspace_bytes.argtypes = [ctypes.POINTER(MoeDesc)]
+        L.afx_moe_block.argtypes = [ctypes.POINTER(MoeDesc), c_void_p, c_void_p, c_int, c_void_p, c_size_t, c_void_p]
         L.afx_mlp_block_noalloc.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_void_p, c_int, c_int, c_int,
                                             c_float, c_int, c_float, c_void_p, c_void_p]
         _lib = L
@@ -388,3 +399,12 @@ def afx_cost_search(chunk_table, hr_table, **kw) -> dict:
     _check("afx_cost_search", lib().afx_cost_search(ctypes.byref(arg), ctypes.byref(out)))
     return dict(sp=out.sp, N=out.N, M_cache=out.M_cache, hr=out.hr, bw_flash_large=out.bw_flash_large,
                 stop_reason=out.stop_reason, cost=out.cost.as_dict())
+
+
+def afx_moe_workspace_bytes(desc: MoeDesc) -> int:
+    return int(lib().afx_moe_workspace_bytes(ctypes.byref(desc)))
+
+
+def afx_moe_block(desc: MoeDesc, x, y, accumulate: int, workspace, workspace_bytes: int, stream=None):
+    _check("afx_moe_block", lib().afx_moe_block(ctypes.byref(desc), _ptr(x), _ptr(y), int(accumulate), _ptr(workspace),
+                                                int(workspace_bytes), _stream(stream)))

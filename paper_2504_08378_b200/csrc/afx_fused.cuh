@@ -14,6 +14,10 @@ enum { IN_X = 0, IN_NORM = 1 };
 
 struct FusedArgs {
     const uint16_t* Wt;
+    // mixture of experts: if wt_table is given, the weights are wt_table[*wt_sel] (both DEVICE;
+    // the choice is made on the device by the router kernel earlier in the stream)
+    const uint16_t* const* wt_table;
+    const int32_t* wt_sel;
     int64_t ldw;
     int K, N, T;
     // ---- input: IN_X reads x; IN_NORM computes x = round(h / rms(h) * gain) ----
@@ -269,6 +273,7 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
         if (side) return;
     }
     AFX_MARK(3);
+    const uint16_t* Wt = a.wt_table != nullptr ? a.wt_table[*a.wt_sel] : a.Wt;
     const int c_lo = s * cnt / S;  // S <= 8, cnt <= 2^20: no overflow
     const int c_hi = (s + 1) * cnt / S;
 
@@ -309,7 +314,7 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
         __syncthreads();
         AFX_MARK(4);
         if (lane_ok)
-            gemv_stream<DT, TMAX, PW, CAP, false>(reinterpret_cast<const uint4*>(a.Wt + out0), T, sm, staged, acc);
+            gemv_stream<DT, TMAX, PW, CAP, false>(reinterpret_cast<const uint4*>(Wt + out0), T, sm, staged, acc);
     }
     AFX_MARK(5);
 

@@ -103,6 +103,7 @@ extern "C" afx_status afx_sparse_gemv(const void* Wt, int dtype, int K, int N, i
     a.ep.y = y;
     a.ep.out_bits = nullptr;
     a.ep.N = N;
+    a.ep.scale = nullptr;
     a.status = dev_status;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     return dtype == AFX_F16 ? launch_gemv<AFX_F16>(a, st) : launch_gemv<AFX_BF16>(a, st);

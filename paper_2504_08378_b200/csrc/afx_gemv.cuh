@@ -61,6 +61,8 @@ struct EpilogueArgs {
     float* y;            // EP_STORE / EP_ACCUM: [T][N] fp32
     uint16_t* out_bits;  // EP_SILU: [T][N/2] 16-bit floats
     int N;               // outputs of the operator (columns of Wt)
+    const float* scale;  // EP_STORE / EP_ACCUM: DEVICE factor applied to the finished sum (an
+                         // expert's routing weight), or NULL for 1
 };
 
 // Streams the staged channels [0, staged) of one tile: acc[t][q] += xv[t][p] * W[row(p)][out0+q].
@@ -188,6 +190,7 @@ __device__ __forceinline__ void gemv_finish_tile(float (&acc)[TMAX][8], int T, i
             }
         }
     }
+    const float out_scale = (EP != EP_SILU && ep.scale != nullptr) ? *ep.scale : 1.0f;
     cluster.sync();  // every contribution has landed
     const float* mine = &recv->v[0];
     if (EP == EP_SILU) {
@@ -214,6 +217,7 @@ __device__ __forceinline__ void gemv_finish_tile(float (&acc)[TMAX][8], int T, i
             if (o < PW && out < ep.N) {
                 float s = 0.0f;
                 for (int q = 0; q < S; ++q) s += mine[(q * T + t) * W + sl];
+                s *= out_scale;
                 float* p = ep.y + static_cast<size_t>(t) * ep.N + out;
                 *p = (EP == EP_ACCUM) ? (e < kGemvThreads ? y_old : *p) + s : s;
             }

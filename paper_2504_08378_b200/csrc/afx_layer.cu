@@ -495,6 +495,142 @@ extern "C" afx_status afx_select_gemv(const void* Wt, int dtype, int K, int N, i
 }
 
 // ---------------------------------------------------------------------------------------------
+// afx_moe_block: dense router + the chosen experts' sparse MLP blocks (Mixtral-shaped layers).
+// ---------------------------------------------------------------------------------------------
+
+namespace afx {
+
+constexpr int kMoeMaxExperts = 16;
+constexpr int kMoeMaxTop = 4;
+constexpr int kMoeThreads = 1024;
+
+struct MoeWork {  // layout of the caller's workspace
+    float logits[kMoeMaxExperts];
+    int32_t sel[kMoeMaxTop];
+    float weight[kMoeMaxTop];
+};
+
+// logits = W_r x over all channels (fp32, fixed order: a thread's channels ascending, lanes by
+// shuffle, warps in warp order), the `top` largest (ties to the lower expert id), softmax over
+// the chosen logits.  One block.
+template <int DT>
+__global__ void __launch_bounds__(kMoeThreads, 1)
+moe_router_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ Wr, int64_t ldr, int K, int E, int top,
+                  MoeWork* __restrict__ w) {
+    __shared__ float part[kMoeThreads / 32][kMoeMaxExperts];
+    float acc[kMoeMaxExperts];
+#pragma unroll
+    for (int e = 0; e < kMoeMaxExperts; ++e) acc[e] = 0.0f;
+    for (int j = threadIdx.x; j < K; j += kMoeThreads) {
+        const float xv = bits_to_float<DT>(x[j]);
+        const uint16_t* row = Wr + static_cast<int64_t>(j) * ldr;
+#pragma unroll
+        for (int e = 0; e < kMoeMaxExperts; ++e)
+            if (e < E) acc[e] = fmaf(xv, bits_to_float<DT>(row[e]), acc[e]);
+    }
+#pragma unroll
+    for (int e = 0; e < kMoeMaxExperts; ++e) {
+        const float v = warp_sum(acc[e]);
+        if (lane_id() == 0) part[warp_id()][e] = v;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float lg[kMoeMaxExperts];
+        for (int e = 0; e < E; ++e) {
+            float s = 0.0f;
+            for (int g = 0; g < kMoeThreads / 32; ++g) s += part[g][e];
+            lg[e] = s;
+            w->logits[e] = s;
+        }
+        uint32_t taken = 0;
+        float chosen[kMoeMaxTop];
+        for (int r = 0; r < top; ++r) {
+            int best = -1;
+            for (int e = 0; e < E; ++e)
+                if (!((taken >> e) & 1u) && (best < 0 || lg[e] > lg[best])) best = e;  // strict >: the lower id wins a tie
+            taken |= 1u << best;
+            w->sel[r] = best;
+            chosen[r] = lg[best];
+        }
+        float z = 0.0f, p[kMoeMaxTop];
+        for (int r = 0; r < top; ++r) {
+            p[r] = expf(chosen[r] - chosen[0]);
+            z += p[r];
+        }
+        for (int r = 0; r < top; ++r) w->weight[r] = p[r] / z;
+    }
+}
+
+}  // namespace afx
+
+extern "C" size_t afx_moe_workspace_bytes(const afx_moe_desc* d) {
+    if (d == nullptr || d->mlp < 8 || d->top < 1 || d->top > afx::kMoeMaxTop) return 0;
+    return afx::align256(sizeof(afx::MoeWork)) + static_cast<size_t>(d->top) * afx::align256(static_cast<size_t>(d->mlp) * 2);
+}
+
+extern "C" afx_status afx_moe_block(const afx_moe_desc* desc, const void* x, float* y, int accumulate, void* workspace,
+                                    size_t workspace_bytes, void* stream) {
+    using namespace afx;
+    if (desc == nullptr || x == nullptr || y == nullptr || workspace == nullptr) return AFX_ERR_INVALID_ARG;
+    const afx_moe_desc& d = *desc;
+    if (d.w_router == nullptr || d.w_gu_table == nullptr || d.w_down_table == nullptr) return AFX_ERR_INVALID_ARG;
+    if (d.hidden < 8 || d.mlp < 8 || d.n_experts < 1 || d.top < 1 || d.top > d.n_experts || d.ld_router < d.n_experts)
+        return AFX_ERR_INVALID_ARG;
+    if (d.n_experts > kMoeMaxExperts || d.top > kMoeMaxTop || d.hidden > kSelectFastMaxK || d.mlp > kSelectFastMaxK)
+        return AFX_ERR_CAPACITY;
+    if (d.dtype != AFX_F16 && d.dtype != AFX_BF16) return AFX_ERR_UNSUPPORTED;
+    if (d.select_mode != AFX_MODE_TOPK && d.select_mode != AFX_MODE_THRESHOLD) return AFX_ERR_UNSUPPORTED;
+    if (d.select_mode == AFX_MODE_TOPK && (d.k_gu < 0 || d.k_gu > d.hidden || d.k_down < 0 || d.k_down > d.mlp))
+        return AFX_ERR_INVALID_ARG;
+    if (d.select_mode == AFX_MODE_THRESHOLD && (d.tau_gu != d.tau_gu || d.tau_down != d.tau_down)) return AFX_ERR_INVALID_ARG;
+    if ((d.hidden & 7) != 0 || (d.mlp & 7) != 0 || !aligned16(y) || (reinterpret_cast<uintptr_t>(x) & 1u) != 0 ||
+        (reinterpret_cast<uintptr_t>(d.w_router) & 1u) != 0 || (reinterpret_cast<uintptr_t>(d.w_gu_table) & 7u) != 0 ||
+        (reinterpret_cast<uintptr_t>(d.w_down_table) & 7u) != 0 || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)
+        return AFX_ERR_ALIGNMENT;
+    if (workspace_bytes < afx_moe_workspace_bytes(desc)) return AFX_ERR_CAPACITY;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    MoeWork* w = static_cast<MoeWork*>(workspace);
+    char* hm_base = static_cast<char*>(workspace) + align256(sizeof(MoeWork));
+    const uint16_t* xb = static_cast<const uint16_t*>(x);
+    const uint16_t* wr = static_cast<const uint16_t*>(d.w_router);
+    if (d.dtype == AFX_F16)
+        moe_router_kernel<AFX_F16><<<1, kMoeThreads, 0, st>>>(xb, wr, d.ld_router, d.hidden, d.n_experts, d.top, w);
+    else
+        moe_router_kernel<AFX_BF16><<<1, kMoeThreads, 0, st>>>(xb, wr, d.ld_router, d.hidden, d.n_experts, d.top, w);
+    if (cudaGetLastError() != cudaSuccess) return AFX_ERR_CUDA;
+    afx_status rc;
+    for (int r = 0; r < d.top; ++r) {
+        uint16_t* hm = reinterpret_cast<uint16_t*>(hm_base + static_cast<size_t>(r) * align256(static_cast<size_t>(d.mlp) * 2));
+        FusedArgs a = {};
+        a.T = 1;
+        a.mode = d.select_mode;
+        a.wt_sel = &w->sel[r];
+        // gate | up of the r-th chosen expert
+        a.wt_table = reinterpret_cast<const uint16_t* const*>(d.w_gu_table);
+        a.ldw = 2 * static_cast<int64_t>(d.mlp);
+        a.K = d.hidden;
+        a.N = 2 * d.mlp;
+        a.x = xb;
+        a.k = d.k_gu;
+        a.tau = d.tau_gu;
+        a.ep = {nullptr, hm, 2 * d.mlp, nullptr};
+        if ((rc = launch_fused<IN_X, EP_SILU>(d.dtype, a, st)) != AFX_OK) return rc;
+        // its down projection, weighted
+        a.wt_table = reinterpret_cast<const uint16_t* const*>(d.w_down_table);
+        a.ldw = d.hidden;
+        a.K = d.mlp;
+        a.N = d.hidden;
+        a.x = hm;
+        a.k = d.k_down;
+        a.tau = d.tau_down;
+        a.ep = {y, nullptr, d.hidden, &w->weight[r]};
+        rc = (accumulate || r > 0) ? launch_fused<IN_X, EP_ACCUM>(d.dtype, a, st) : launch_fused<IN_X, EP_STORE>(d.dtype, a, st);
+        if (rc != AFX_OK) return rc;
+    }
+    return AFX_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
 // afx_mlp_block_noalloc: the MLP block for callers that cannot allocate device memory.
 // ---------------------------------------------------------------------------------------------
 
