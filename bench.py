@@ -474,6 +474,8 @@ def run_afx(args):
         variants["config1_single_projection"] = variant_config1(st)
         variants["config2_mlp_block_7b_threshold_sweep"] = variant_config2(st)
         variants["config4_llama13b_step"] = variant_config4(st)
+        variants["mixtral_shaped_moe_block"] = variant_moe(st)
+        torch.cuda.empty_cache()
         variants["config5_llama70b_host_weights_cache"] = cache70b_measure(2, 64, st)
         variants["config5_cross_layer_group_preload"] = swap70b_measure(4, 3, groups=(0, 2), st=st)
         variants["cost_model"] = cost_model_report(peak, variants["config5_cross_layer_group_preload"],
@@ -983,6 +985,56 @@ def swap70b_measure(n_layers, tokens, groups=(0, 1, 2, 4), st=None, lead="first"
             "speedup_over_serial": {kk: round(base / v["ms_per_token"], 3) for kk, v in results.items()} if base else None,
             "paper_context": "the paper reports 4.1x at 4 layers per group over serial loading on phone flash, where small "
                              "reads are far slower than large ones (Sec. 7.3)"}
+
+
+def variant_moe(st, n_layers=4):
+    """Mixtral-8x7B-shaped expert layers (hidden 4096, expert MLP 14336, 8 experts, 2 per token,
+    bf16, random-init): the dense router plus the two chosen experts' sparse MLP blocks at 50 %
+    top-k, on Laplace inputs; distinct layers in rotation (11 GB of expert weights, far beyond
+    L2).  Shapes only: routing of random weights is near uniform."""
+    import numpy as np
+    import torch
+    from paper_2504_08378_b200 import afx, synth
+    dt, H, M, E, top = "bf16", 4096, 14336, 8, 2
+    k_gu, k_down = synth.keep_count(H, 50), synth.keep_count(M, 50)
+    descs, keep = [], []
+    for l in range(n_layers):
+        gu = [synth.device_normal_bits(7, 1000 * (l + 1) + 10 * e + 1, (H, 2 * M), 0.02, dt) for e in range(E)]
+        down = [synth.device_normal_bits(7, 1000 * (l + 1) + 10 * e + 2, (M, H), 0.02, dt) for e in range(E)]
+        wr = synth.device_normal_bits(7, 1000 * (l + 1) + 99, (H, E), 0.05, dt)
+        gt = torch.tensor([t.data_ptr() for t in gu], dtype=torch.int64, device="cuda")
+        dtab = torch.tensor([t.data_ptr() for t in down], dtype=torch.int64, device="cuda")
+        keep.append((gu, down, wr, gt, dtab))
+        descs.append(afx.MoeDesc(dtype=afx.DTYPES[dt], hidden=H, mlp=M, n_experts=E, top=top, select_mode=afx.MODE_TOPK,
+                                 k_gu=k_gu, k_down=k_down, tau_gu=0.0, tau_down=0.0, w_router=wr.data_ptr(), ld_router=E,
+                                 w_gu_table=gt.data_ptr(), w_down_table=dtab.data_ptr()))
+    nbytes = afx.afx_moe_workspace_bytes(descs[0])
+    raw = torch.zeros(nbytes + 256, dtype=torch.uint8, device="cuda")
+    ws = raw[(-raw.data_ptr()) % 256:][:nbytes]
+    xs = [torch.from_numpy(synth.laplace_bits(7, 100 + i, (1, H), dt).view(np.int16)).cuda() for i in range(16)]
+    y = torch.zeros((1, H), dtype=torch.float32, device="cuda")
+    g = torch.cuda.CUDAGraph()
+    n = 16
+    with torch.cuda.stream(st):
+        afx.afx_moe_block(descs[0], xs[0], y, 1, ws, nbytes, stream=st)
+        st.synchronize()
+        with torch.cuda.graph(g, stream=st):
+            for i in range(n):
+                afx.afx_moe_block(descs[i % n_layers], xs[i], y, 1, ws, nbytes, stream=st)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for _ in range(3):
+            g.replay()
+        e0.record(st)
+        reps = 10
+        for _ in range(reps):
+            g.replay()
+        e1.record(st)
+    e1.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / (reps * n)
+    nbytes_active = top * 2 * (k_gu * 2 * M + k_down * H)
+    return {"workload": "mixtral8x7b_shaped_moe_block_bf16_top2of8_sparsity50", "layers_in_rotation": n_layers,
+            "us_per_block": round(us, 2), "kernels_per_block": 1 + 2 * top, "active_expert_bytes": nbytes_active,
+            "gbs": round(nbytes_active / (us * 1e-6) / 1e9, 1)}
 
 
 def cost_model_report(hbm_gbs, swap, cache):

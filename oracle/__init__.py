@@ -288,3 +288,34 @@ def cost_model(sp, hr, si, N, S_l, bw_mem, bw_flash_small, bw_flash_large, M_cac
         groups = -(-n_layers // N)
         out["T_token"] = T_load + (groups - 1) * T_overlap + T_comp
     return out
+
+
+# ---- 4-bit block-quantised weights (Sec. 6: the channel's scales travel with the channel) ----
+
+def q4_decode(rows, N: int) -> np.ndarray:
+    """fp64 values [K][N] of channel-contiguous 4-bit rows: per channel N/2 bytes of codes, then
+    N/32 fp16 scales; block b = outputs 32b .. 32b+31, byte m of the block holds the code of
+    output 32b + m in its low 4 bits and of output 32b + 16 + m in its high 4 bits; value =
+    (code - 8) * scale.  Plain loops over that definition."""
+    rows = np.ascontiguousarray(rows, np.uint8)
+    K = rows.shape[0]
+    out = np.empty((K, N), np.float64)
+    for j in range(K):
+        scales = decode(rows[j, N // 2: N // 2 + N // 16].copy().view(np.uint16), "f16")
+        for b in range(N // 32):
+            blk = rows[j, 16 * b: 16 * b + 16]
+            for m in range(16):
+                out[j, 32 * b + m] = (int(blk[m] & 0x0F) - 8) * scales[b]
+                out[j, 32 * b + 16 + m] = (int(blk[m] >> 4) - 8) * scales[b]
+    return out
+
+
+def sparse_gemv_q4(rows, N: int, x, dtype: str, idx) -> np.ndarray:
+    """y[N] (fp64) = sum_c x[idx[c]] * W[idx[c]][:], W = q4_decode(rows), ascending c."""
+    xv = decode(np.asarray(x, np.uint16).reshape(-1), dtype)
+    idx = np.asarray(idx, np.int64)
+    W = q4_decode(np.asarray(rows)[idx], N) if idx.size else np.zeros((0, N))
+    y = np.zeros(N)
+    for c in range(idx.size):
+        y += xv[idx[c]] * W[c]
+    return y[None, :]

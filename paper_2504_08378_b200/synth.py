@@ -201,3 +201,28 @@ def split_gate_up(w_gu: np.ndarray):
     v = w_gu.reshape(K, N2 // 16, 2, 8)
     return (np.ascontiguousarray(v[:, :, 0, :]).reshape(K, N2 // 2),
             np.ascontiguousarray(v[:, :, 1, :]).reshape(K, N2 // 2))
+
+
+# ---- 4-bit block-quantised weights (the storage type the paper evaluates) ----
+
+def q4_row_bytes(N: int) -> int:
+    """Bytes of one channel of N outputs (N a multiple of 32) in the 4-bit layout: N/2 bytes of
+    4-bit codes, then N/32 fp16 block scales, padded to a multiple of 16 bytes."""
+    assert N % 32 == 0
+    return (N // 2 + N // 16 + 15) // 16 * 16
+
+
+def q4_weight(seed: int, stream: int, K: int, N: int, sigma: float = 0.02) -> np.ndarray:
+    """Random-init channel-contiguous 4-bit weights, drawn directly in storage form: uint8
+    [K][q4_row_bytes(N)].  Each block of 32 outputs has an fp16 scale d and 32 codes q in 0..15
+    (value (q - 8) * d); codes are rounded normal draws with the spread a quantised N(0, sigma^2)
+    block has (its largest magnitude lands near code 0 or 15), scales scatter around
+    2.5 * sigma / 8.  Byte m of a block holds code m (low 4 bits) and code m + 16 (high 4 bits)."""
+    g = rng(seed, stream)
+    q = np.clip(np.rint(g.standard_normal((K, N // 32, 32), dtype=np.float32) * (8.0 / 2.5) + 8.0), 0, 15).astype(np.uint8)
+    d = (sigma * 2.5 / 8.0 * (1.0 + 0.1 * g.standard_normal((K, N // 32), dtype=np.float32)))
+    d *= np.where(g.random((K, N // 32)) < 0.5, -1.0, 1.0).astype(np.float32)   # the format allows negative scales
+    rows = np.zeros((K, q4_row_bytes(N)), np.uint8)
+    rows[:, : N // 2] = (q[:, :, :16] | (q[:, :, 16:] << 4)).reshape(K, N // 2)
+    rows[:, N // 2: N // 2 + N // 16] = d.astype(np.float16).view(np.uint8).reshape(K, N // 16)
+    return rows
