@@ -474,6 +474,7 @@ def run_afx(args):
         variants["config1_single_projection"] = variant_config1(st)
         variants["config2_mlp_block_7b_threshold_sweep"] = variant_config2(st)
         variants["config4_llama13b_step"] = variant_config4(st)
+        variants["q4_sparse_gemv"] = variant_q4(st, peak)
         variants["mixtral_shaped_moe_block"] = variant_moe(st)
         torch.cuda.empty_cache()
         variants["config5_llama70b_host_weights_cache"] = cache70b_measure(2, 64, st)
@@ -1035,6 +1036,59 @@ def variant_moe(st, n_layers=4):
     return {"workload": "mixtral8x7b_shaped_moe_block_bf16_top2of8_sparsity50", "layers_in_rotation": n_layers,
             "us_per_block": round(us, 2), "kernels_per_block": 1 + 2 * top, "active_expert_bytes": nbytes_active,
             "gbs": round(nbytes_active / (us * 1e-6) / 1e9, 1)}
+
+
+def variant_q4(st, peak):
+    """afx_sparse_gemv_q4 (4-bit codes + fp16 block scales per channel, the storage type the
+    paper evaluates) at the 7B operator shapes, top 50 % of the channels, 32 distinct matrices
+    per shape in rotation.  Bytes = active rows * row bytes (codes and scales)."""
+    import numpy as np
+    import torch
+    from paper_2504_08378_b200 import afx, synth
+    out = {"note": "about 2.3 instructions per weight: bound by instruction issue before HBM"}
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(77)
+    for name, K, N in (("gate_up", 4096, 22016), ("qkv", 4096, 12288), ("down", 11008, 4096), ("o", 4096, 4096)):
+        rb = afx.afx_q4_row_bytes(N)
+        n_mat = 32
+        mats = []
+        for i in range(n_mat):  # random codes; scales near 0.006 (input generation)
+            m = torch.randint(0, 256, (K, rb), generator=gen, device="cuda", dtype=torch.uint8)
+            sc = (0.00625 * (1 + 0.1 * torch.randn((K, N // 32), generator=gen, device="cuda"))).to(torch.float16)
+            m[:, N // 2: N // 2 + N // 16] = sc.view(torch.uint8)
+            mats.append(m)
+        k = synth.keep_count(K, 50)
+        xs = [torch.from_numpy(synth.laplace_bits(8, 100 + i, (1, K), "bf16").view(np.int16)).cuda() for i in range(4)]
+        idxs, cnt = [], torch.tensor([k], dtype=torch.int32, device="cuda")
+        for x in xs:
+            idx = torch.empty(K, dtype=torch.int32, device="cuda")
+            afx.afx_select_active(x, "bf16", K, 1, afx.MODE_TOPK, k, 0.0, idx, torch.zeros(1, dtype=torch.int32, device="cuda"), None)
+            idxs.append(idx)
+        y = torch.empty(N, dtype=torch.float32, device="cuda")
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(st):
+            afx.afx_sparse_gemv_q4(mats[0], K, N, rb, xs[0], "bf16", idxs[0], cnt, y, 0, stream=st)
+            st.synchronize()
+            with torch.cuda.graph(g, stream=st):
+                for i in range(n_mat):
+                    afx.afx_sparse_gemv_q4(mats[i], K, N, rb, xs[i % 4], "bf16", idxs[i % 4], cnt, y, 0, stream=st)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            for _ in range(3):
+                g.replay()
+            e0.record(st)
+            reps = 10
+            for _ in range(reps):
+                g.replay()
+            e1.record(st)
+        e1.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / (reps * n_mat)
+        nbytes = k * rb
+        out[name] = {"K": K, "N": N, "k": k, "us_per_launch": round(us, 2), "bytes": nbytes,
+                     "gbs": round(nbytes / (us * 1e-6) / 1e9, 1), "frac_of_measured_hbm": round(nbytes / (us * 1e-6) / 1e9 / peak, 4),
+                     "weights_per_us": round(k * N / us / 1e6, 2)}
+        del mats
+        torch.cuda.empty_cache()
+    return out
 
 
 def cost_model_report(hbm_gbs, swap, cache):

@@ -151,6 +151,25 @@ afx_status afx_select_gemv(const void* Wt, int dtype, int K, int N, int64_t ldw,
                            int mode, int k, float tau, float* y, int accumulate, int32_t* idx_out,
                            int32_t* count_out, int32_t* kth_hint, void* stream);
 
+/*
+ * The same sparse GEMV over 4-bit block-quantised weights (the storage type of every model the
+ * paper evaluates, Sec. 7.1; Sec. 6: the weights are transposed so that a channel's scaling
+ * factors are read together with the channel).  Channel j is the row Wq[j * ldq_bytes ..):
+ * N/2 bytes of 4-bit codes, then N/32 fp16 scales; a block of 32 outputs b has 16 code bytes --
+ * byte m holds the code of output 32b + m in its low 4 bits and of output 32b + 16 + m in its
+ * high 4 bits -- and one scale; value = (code - 8) * scale (the block format of llama.cpp's
+ * 4-bit type with the scales moved behind the codes, so that both parts keep 16-byte alignment).
+ *
+ *   Wq         DEVICE, 16-byte aligned; N % 32 == 0; ldq_bytes % 16 == 0, >= afx_q4_row_bytes(N).
+ *   x          DEVICE [K] 16-bit floats of type x_dtype (one token).
+ *   idx,count,dev_status   as for afx_sparse_gemv;  y DEVICE [N] fp32.
+ * fp32 accumulation in a fixed order.
+ */
+size_t afx_q4_row_bytes(int N); /* bytes of one channel row without padding beyond 16 (0: bad N) */
+afx_status afx_sparse_gemv_q4(const void* Wq, int K, int N, int64_t ldq_bytes, const void* x, int x_dtype,
+                              const int32_t* idx, const int32_t* count, float* y, int accumulate,
+                              int32_t* dev_status, void* stream);
+
 /* ------------------------------------------------------------------------------------------
  * Decoder layers: every linear operator of a Llama-shaped layer run as ONE kernel that
  * normalises (where the layer does), selects the active channels of its own input and

@@ -292,11 +292,11 @@ def cost_model(sp, hr, si, N, S_l, bw_mem, bw_flash_small, bw_flash_large, M_cac
 
 # ---- 4-bit block-quantised weights (Sec. 6: the channel's scales travel with the channel) ----
 
-def q4_decode(rows, N: int) -> np.ndarray:
+def q4_decode_loops(rows, N: int) -> np.ndarray:
     """fp64 values [K][N] of channel-contiguous 4-bit rows: per channel N/2 bytes of codes, then
     N/32 fp16 scales; block b = outputs 32b .. 32b+31, byte m of the block holds the code of
     output 32b + m in its low 4 bits and of output 32b + 16 + m in its high 4 bits; value =
-    (code - 8) * scale.  Plain loops over that definition."""
+    (code - 8) * scale.  Plain loops over that definition (small inputs)."""
     rows = np.ascontiguousarray(rows, np.uint8)
     K = rows.shape[0]
     out = np.empty((K, N), np.float64)
@@ -308,6 +308,17 @@ def q4_decode(rows, N: int) -> np.ndarray:
                 out[j, 32 * b + m] = (int(blk[m] & 0x0F) - 8) * scales[b]
                 out[j, 32 * b + 16 + m] = (int(blk[m] >> 4) - 8) * scales[b]
     return out
+
+
+def q4_decode(rows, N: int) -> np.ndarray:
+    """The same decoding with whole-array numpy operations (for inputs of real size; the tests
+    hold it equal to q4_decode_loops)."""
+    rows = np.ascontiguousarray(rows, np.uint8)
+    K = rows.shape[0]
+    codes = rows[:, : N // 2].reshape(K, N // 32, 16)
+    q = np.concatenate([codes & 0x0F, codes >> 4], axis=2).astype(np.float64)     # [K][block][32]
+    scales = decode(rows[:, N // 2: N // 2 + N // 16].copy().view(np.uint16), "f16")  # [K][block]
+    return ((q - 8.0) * scales[:, :, None]).reshape(K, N)
 
 
 def sparse_gemv_q4(rows, N: int, x, dtype: str, idx) -> np.ndarray:

@@ -170,6 +170,10 @@ def lib() -> ctypes.CDLL:
         L.afx_moe_workspace_bytes.restype = c_size_t
         L.afx_moe_workspace_bytes.argtypes = [ctypes.POINTER(MoeDesc)]
         L.afx_moe_block.argtypes = [ctypes.POINTER(MoeDesc), c_void_p, c_void_p, c_int, c_void_p, c_size_t, c_void_p]
+        L.afx_q4_row_bytes.restype = c_size_t
+        L.afx_q4_row_bytes.argtypes = [c_int]
+        L.afx_sparse_gemv_q4.argtypes = [c_void_p, c_int, c_int, c_int64, c_void_p, c_int, c_void_p, c_void_p, c_void_p,
+                                         c_int, c_void_p, c_void_p]
         L.afx_mlp_block_noalloc.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_void_p, c_int, c_int, c_int,
                                             c_float, c_int, c_float, c_void_p, c_void_p]
         _lib = L
@@ -408,3 +412,14 @@ def afx_moe_workspace_bytes(desc: MoeDesc) -> int:
 def afx_moe_block(desc: MoeDesc, x, y, accumulate: int, workspace, workspace_bytes: int, stream=None):
     _check("afx_moe_block", lib().afx_moe_block(ctypes.byref(desc), _ptr(x), _ptr(y), int(accumulate), _ptr(workspace),
                                                 int(workspace_bytes), _stream(stream)))
+
+
+def afx_q4_row_bytes(N: int) -> int:
+    return int(lib().afx_q4_row_bytes(int(N)))
+
+
+def afx_sparse_gemv_q4(Wq, K: int, N: int, ldq_bytes: int, x, x_dtype, idx, count, y, accumulate: int, stream=None,
+                       dev_status=None):
+    _check("afx_sparse_gemv_q4",
+           lib().afx_sparse_gemv_q4(_ptr(Wq), int(K), int(N), int(ldq_bytes), _ptr(x), _dt(x_dtype), _ptr(idx), _ptr(count),
+                                    _ptr(y), int(accumulate), _ptr(dev_status), _stream(stream)))

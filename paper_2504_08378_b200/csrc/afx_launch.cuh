@@ -38,10 +38,10 @@ inline bool ensure_dyn_smem(const void* kern, size_t dyn_smem) {
     return true;
 }
 
-// How many clusters of S blocks of `kern` (kGemvThreads threads, dyn_smem bytes of dynamic
-// shared memory) the current device keeps resident at once.  Cached per (device, kernel, S,
+// How many clusters of S blocks of `kern` (`threads` threads, dyn_smem bytes of dynamic shared
+// memory) the current device keeps resident at once.  Cached per (device, kernel, S,
 // dyn_smem).  Returns 0 if the query fails.
-inline int max_active_clusters(const void* kern, int S, size_t dyn_smem) {
+inline int max_active_clusters(const void* kern, int S, size_t dyn_smem, int threads = kGemvThreads) {
     struct Entry {
         int dev;
         const void* kern;
@@ -59,7 +59,7 @@ inline int max_active_clusters(const void* kern, int S, size_t dyn_smem) {
     ensure_dyn_smem(kern, dyn_smem);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(S, 1, 1);
-    cfg.blockDim = dim3(kGemvThreads, 1, 1);
+    cfg.blockDim = dim3(threads, 1, 1);
     cfg.dynamicSmemBytes = dyn_smem;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -130,14 +130,14 @@ inline GemvShapeChoice choose_gemv_shape(int N, const void* const kerns[3], size
 // the work already in the stream.
 template <class Kern, class Args>
 inline afx_status launch_clustered(Kern kern, int S, int tiles, size_t dyn_smem, const Args& a,
-                                   cudaStream_t st) {
+                                   cudaStream_t st, int threads = kGemvThreads) {
     if (!ensure_dyn_smem(reinterpret_cast<const void*>(kern), dyn_smem)) {
         cudaGetLastError();
         return AFX_ERR_CUDA;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(S, tiles, 1);
-    cfg.blockDim = dim3(kGemvThreads, 1, 1);
+    cfg.blockDim = dim3(threads, 1, 1);
     cfg.dynamicSmemBytes = dyn_smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[2];

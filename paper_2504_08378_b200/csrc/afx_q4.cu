@@ -1,0 +1,257 @@
+// afx_sparse_gemv_q4: sparse GEMV over 4-bit block-quantised, channel-contiguous weights
+// (Sec. 6: the weights are stored transposed so that a channel's scaling factors are read with
+// the channel; Sec. 7.1: every evaluated model is 4-bit).
+//
+// A channel's row is [N/2 bytes of 4-bit codes][N/32 fp16 scales]; a block of 32 outputs is 16
+// bytes of codes and one scale: byte m = code of output m (low 4 bits) and of output 16 + m
+// (high 4 bits); value = (code - 8) * scale.  One lane owns one block of one channel per load:
+// a 16-byte read of the codes plus the block's scale, x * scale once, then 32 multiply-adds with
+// the codes turned into fp32 by a byte permute into the mantissa of 2^23 (0x4B0000qq = 2^23 + q)
+// and one subtraction of 2^23 + 8 -- two-wide adds and fused multiply-adds.  The tile of a
+// cluster is LPC blocks (LPC * 32 outputs) wide; the S blocks of the cluster split the active
+// list and meet through distributed shared memory in rank order; sums are fp32 in a fixed
+// order.  4x fewer bytes per weight than the 16-bit kernels, about 2.3 instructions per weight:
+// this kernel is bound by instruction issue before it is bound by HBM.
+#include <cooperative_groups.h>
+
+#include "afx_launch.cuh"
+
+namespace afx {
+
+namespace cg = cooperative_groups;
+
+constexpr int kQ4Threads = 512;
+constexpr int kQ4Warps = kQ4Threads / 32;
+constexpr int kQ4Unroll = 4;   // 16-byte loads in flight per lane
+constexpr int kQ4Cap = 1024;   // staged list entries per pass
+
+struct Q4Args {
+    const unsigned char* Wq;
+    int64_t ldq;  // row stride in bytes (multiple of 16)
+    int K, N;
+    const uint16_t* x;
+    const int32_t* idx;
+    const int32_t* count;
+    float* y;
+    int accumulate;
+    int32_t* status;
+};
+
+// (code - 8) for the four codes in the low nibbles of v's bytes, as two fp32 pairs.
+__device__ __forceinline__ void nibbles_to_pairs(uint32_t v, f32x2& p01, f32x2& p23) {
+    const uint32_t magic = 0x4B000000u;  // 2^23: the low mantissa byte becomes the code
+    const float bias = 8388616.0f;       // 2^23 + 8
+    const float f0 = __uint_as_float(__byte_perm(v, magic, 0x7540)) - bias;
+    const float f1 = __uint_as_float(__byte_perm(v, magic, 0x7541)) - bias;
+    const float f2 = __uint_as_float(__byte_perm(v, magic, 0x7542)) - bias;
+    const float f3 = __uint_as_float(__byte_perm(v, magic, 0x7543)) - bias;
+    p01 = pack_f32x2(f0, f1);
+    p23 = pack_f32x2(f2, f3);
+}
+
+// LPC lanes (blocks of 32 outputs) per channel piece: tile = LPC * 32 outputs.
+template <int XDT, int LPC>
+__global__ void __launch_bounds__(kQ4Threads, 1) sparse_gemv_q4_kernel(Q4Args a) {
+    constexpr int SUB = 32 / LPC;        // channels per warp-wide load
+    constexpr int EG = kQ4Warps * SUB;   // channel groups of the block
+    constexpr int PW = LPC * 32;         // outputs of the tile
+    extern __shared__ __align__(16) unsigned char q4_dyn[];
+    uint32_t* s_off = reinterpret_cast<uint32_t*>(q4_dyn);          // [kQ4Cap] row offset in 16-byte units
+    float* s_x = reinterpret_cast<float*>(s_off + kQ4Cap);          // [kQ4Cap]
+    float* s_red = s_x + kQ4Cap;                                    // [kQ4Warps][PW] then part[PW]
+    __shared__ int first_ok;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int S = static_cast<int>(cluster.num_blocks());
+    const int rank = static_cast<int>(cluster.block_rank());
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tile = blockIdx.y;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    int cnt = *a.count;
+    if (cnt < 0 || cnt > a.K) {
+        if (tid == 0 && rank == 0 && tile == 0) report_status(a.status, AFX_ERR_CAPACITY);
+        cnt = max(0, min(cnt, a.K));
+    }
+    const int c_lo = static_cast<int>(static_cast<int64_t>(rank) * cnt / S);
+    const int c_hi = static_cast<int>(static_cast<int64_t>(rank + 1) * cnt / S);
+    const int blk = tile * LPC + (lane % LPC);  // this lane's block of 32 outputs
+    const bool lane_ok = blk * 32 < a.N;
+    const uint64_t ld16 = static_cast<uint64_t>(a.ldq >> 4);
+    const uint4* codes = reinterpret_cast<const uint4*>(a.Wq) + blk;                        // + row offset
+    const uint16_t* scales = reinterpret_cast<const uint16_t*>(a.Wq + (a.N >> 1)) + blk;    // + row offset * 8
+    const int eg = warp * SUB + lane / LPC;
+
+    f32x2 acc[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) acc[i] = pack_f32x2(0.0f, 0.0f);
+
+    for (int c0 = c_lo; c0 < c_hi; c0 += kQ4Cap) {
+        int staged = min(kQ4Cap, c_hi - c0);
+        __syncthreads();
+        bool skipped = false;
+        for (int i = tid; i < staged; i += kQ4Threads) {
+            const int j = a.idx[c0 + i];
+            const uint64_t off = static_cast<uint64_t>(j < 0 ? 0 : j) * ld16;
+            const bool ok = static_cast<unsigned>(j) < static_cast<unsigned>(a.K) && off + ld16 <= 0xFFFFFFFFull;
+            if (!ok && tile == 0) report_status(a.status, AFX_ERR_INVALID_ARG);
+            skipped |= !ok;
+            s_off[i] = ok ? static_cast<uint32_t>(off) : 0xFFFFFFFFu;
+            s_x[i] = ok ? bits_to_float<XDT>(a.x[j]) : 0.0f;
+        }
+        if (__syncthreads_or(skipped)) {  // rare: a skipped entry reads the row of one that takes part
+            if (tid == 0) first_ok = staged;
+            __syncthreads();
+            for (int i = tid; i < staged; i += kQ4Threads)
+                if (s_off[i] != 0xFFFFFFFFu) atomicMin(&first_ok, i);
+            __syncthreads();
+            const int f = first_ok;
+            if (f < staged) {
+                const uint32_t safe = s_off[f];
+                __syncthreads();
+                for (int i = tid; i < staged; i += kQ4Threads)
+                    if (s_off[i] == 0xFFFFFFFFu) s_off[i] = safe;
+            } else {
+                staged = 0;
+            }
+            __syncthreads();
+        }
+        if (lane_ok) {
+            for (int p = eg; p < staged; p += EG * kQ4Unroll) {
+                uint4 raw[kQ4Unroll];
+                uint16_t sc[kQ4Unroll];
+#pragma unroll
+                for (int u = 0; u < kQ4Unroll; ++u) {
+                    const int pp = p + u * EG;
+                    if (pp < staged) {
+                        const uint32_t off = s_off[pp];
+                        raw[u] = ld_stream_16B(codes + off);
+                        sc[u] = __ldg(scales + static_cast<size_t>(off) * 8);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < kQ4Unroll; ++u) {
+                    const int pp = p + u * EG;
+                    if (pp < staged) {
+                        const float s = s_x[pp] * __half2float(__ushort_as_half(sc[u]));
+                        const f32x2 s2 = pack_f32x2(s, s);
+                        const uint32_t w[4] = {raw[u].x, raw[u].y, raw[u].z, raw[u].w};
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {  // word q: outputs 4q..4q+3 (low nibbles), 16+4q.. (high)
+                            f32x2 a01, a23;
+                            nibbles_to_pairs(w[q] & 0x0F0F0F0Fu, a01, a23);
+                            fma_f32x2(acc[2 * q], a01, s2);
+                            fma_f32x2(acc[2 * q + 1], a23, s2);
+                            nibbles_to_pairs((w[q] >> 4) & 0x0F0F0F0Fu, a01, a23);
+                            fma_f32x2(acc[8 + 2 * q], a01, s2);
+                            fma_f32x2(acc[8 + 2 * q + 1], a23, s2);
+                        }
+                    }
+                }
+            }
+        }
+    }
+    // ---- lane groups of a warp, warps of the block, blocks of the cluster: fixed order ----
+    float v[32];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) unpack_f32x2(acc[i], v[2 * i], v[2 * i + 1]);
+#pragma unroll
+    for (int o = LPC; o < 32; o <<= 1)
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] += __shfl_xor_sync(0xFFFFFFFFu, v[i], o);
+    __syncthreads();
+    if (lane < LPC) {
+        float4* d4 = reinterpret_cast<float4*>(s_red + warp * PW + lane * 32);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) d4[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+    }
+    __syncthreads();
+    float* part = s_red + kQ4Warps * PW;  // this block's sums, read by the cluster
+    for (int o = tid; o < PW; o += kQ4Threads) {
+        float s = 0.0f;
+#pragma unroll
+        for (int g = 0; g < kQ4Warps; ++g) s += s_red[g * PW + o];
+        part[o] = s;
+    }
+    cluster.sync();
+    for (int o = rank + S * tid; o < PW; o += S * kQ4Threads) {
+        const int out = tile * PW + o;
+        if (out < a.N) {
+            float s = 0.0f;
+            for (int q = 0; q < S; ++q) s += cluster.map_shared_rank(part, q)[o];
+            a.y[out] = a.accumulate ? a.y[out] + s : s;
+        }
+    }
+    cluster.sync();  // peers may still be reading this block's sums
+}
+
+static size_t q4_dyn_smem(int lpc) {
+    return static_cast<size_t>(kQ4Cap) * 8 + static_cast<size_t>(kQ4Warps + 1) * lpc * 32 * 4;
+}
+
+template <int XDT>
+static afx_status launch_q4(const Q4Args& a, cudaStream_t st) {
+    const void* kerns[3] = {reinterpret_cast<const void*>(sparse_gemv_q4_kernel<XDT, 32>),
+                            reinterpret_cast<const void*>(sparse_gemv_q4_kernel<XDT, 8>),
+                            reinterpret_cast<const void*>(sparse_gemv_q4_kernel<XDT, 4>)};
+    const int lpcs[3] = {32, 8, 4};
+    // the widest tile and largest cluster that keep every cluster resident at once, most blocks wins
+    int best = 2, best_S = 1, best_blocks = -1;
+    for (int i = 0; i < 3; ++i) {
+        const int tiles = (a.N + lpcs[i] * 32 - 1) / (lpcs[i] * 32);
+        const size_t dyn = q4_dyn_smem(lpcs[i]);
+        for (int S = kMaxCluster; S >= 1; --S) {
+            const int margin = (tiles + 15) / 16 < 2 ? 2 : (tiles + 15) / 16;
+            if (max_active_clusters(kerns[i], S, dyn, kQ4Threads) >= tiles + margin) {
+                if (tiles * S > best_blocks) {
+                    best_blocks = tiles * S;
+                    best = i;
+                    best_S = S;
+                }
+                break;
+            }
+        }
+    }
+    const int lpc = lpcs[best];
+    const int tiles = (a.N + lpc * 32 - 1) / (lpc * 32);
+    if (tiles > 65535) return AFX_ERR_CAPACITY;
+    const size_t dyn = q4_dyn_smem(lpc);
+    switch (lpc) {
+        case 32: return launch_clustered(sparse_gemv_q4_kernel<XDT, 32>, best_S, tiles, dyn, a, st, kQ4Threads);
+        case 8: return launch_clustered(sparse_gemv_q4_kernel<XDT, 8>, best_S, tiles, dyn, a, st, kQ4Threads);
+        default: return launch_clustered(sparse_gemv_q4_kernel<XDT, 4>, best_S, tiles, dyn, a, st, kQ4Threads);
+    }
+}
+
+}  // namespace afx
+
+extern "C" size_t afx_q4_row_bytes(int N) {
+    if (N < 32 || (N & 31) != 0) return 0;
+    return (static_cast<size_t>(N) / 2 + static_cast<size_t>(N) / 16 + 15) / 16 * 16;
+}
+
+extern "C" afx_status afx_sparse_gemv_q4(const void* Wq, int K, int N, int64_t ldq_bytes, const void* x, int x_dtype,
+                                         const int32_t* idx, const int32_t* count, float* y, int accumulate,
+                                         int32_t* dev_status, void* stream) {
+    using namespace afx;
+    if (Wq == nullptr || x == nullptr || idx == nullptr || count == nullptr || y == nullptr) return AFX_ERR_INVALID_ARG;
+    if (K <= 0 || N <= 0) return AFX_ERR_INVALID_ARG;
+    if (x_dtype != AFX_F16 && x_dtype != AFX_BF16) return AFX_ERR_UNSUPPORTED;
+    if ((N & 31) != 0 || (ldq_bytes & 15) != 0 || !aligned16(Wq) || (reinterpret_cast<uintptr_t>(y) & 3u) != 0 ||
+        (reinterpret_cast<uintptr_t>(x) & 1u) != 0 || (reinterpret_cast<uintptr_t>(idx) & 3u) != 0 ||
+        (reinterpret_cast<uintptr_t>(count) & 3u) != 0 || (reinterpret_cast<uintptr_t>(dev_status) & 3u) != 0)
+        return AFX_ERR_ALIGNMENT;
+    if (ldq_bytes < static_cast<int64_t>(afx_q4_row_bytes(N))) return AFX_ERR_INVALID_ARG;
+    Q4Args a;
+    a.Wq = static_cast<const unsigned char*>(Wq);
+    a.ldq = ldq_bytes;
+    a.K = K;
+    a.N = N;
+    a.x = static_cast<const uint16_t*>(x);
+    a.idx = idx;
+    a.count = count;
+    a.y = y;
+    a.accumulate = accumulate ? 1 : 0;
+    a.status = dev_status;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return x_dtype == AFX_F16 ? launch_q4<AFX_F16>(a, st) : launch_q4<AFX_BF16>(a, st);
+}

@@ -11,7 +11,8 @@ def test_q4_decode_hand_block():
     row = np.zeros((1, synth.q4_row_bytes(32)), np.uint8)
     row[0, :16] = [m | ((15 - m) << 4) for m in range(16)]
     row[0, 16:18] = np.array([0.5], np.float16).view(np.uint8)
-    w = oracle.q4_decode(row, 32)[0]
+    w = oracle.q4_decode_loops(row, 32)[0]
+    assert np.array_equal(w, oracle.q4_decode(row, 32)[0])
     assert w[:16].tolist() == [(m - 8) / 2 for m in range(16)]
     assert w[16:].tolist() == [(7 - m) / 2 for m in range(16)]
     # y = x * W for a single active channel
@@ -27,6 +28,7 @@ def test_q4_decode_equals_a_vectorised_numpy_decode():
     q = np.concatenate([codes & 0x0F, codes >> 4], axis=2).astype(np.float64)          # [K][blocks][32]
     d = rows[:, N // 2: N // 2 + N // 16].copy().view(np.float16).astype(np.float64)   # [K][blocks]
     want = ((q - 8.0) * d[:, :, None]).reshape(K, N)
+    assert np.array_equal(oracle.q4_decode_loops(rows, N), want)
     assert np.array_equal(oracle.q4_decode(rows, N), want)
     assert 0 < np.abs(want).max() < 0.1 and np.unique(codes & 0x0F).size == 16
 
