@@ -10,8 +10,9 @@
 // and one subtraction of 2^23 + 8 -- two-wide adds and fused multiply-adds.  The tile of a
 // cluster is LPC blocks (LPC * 32 outputs) wide; the S blocks of the cluster split the active
 // list and meet through distributed shared memory in rank order; sums are fp32 in a fixed
-// order.  4x fewer bytes per weight than the 16-bit kernels, about 2.3 instructions per weight:
-// this kernel is bound by instruction issue before it is bound by HBM.
+// order.  3.5x fewer bytes per weight than the 16-bit kernels, but about 5 executed
+// instructions per weight: this kernel is bound by instruction issue (one 512-thread block of
+// 120+ registers per SM), not by HBM.
 #include <cooperative_groups.h>
 
 #include "afx_launch.cuh"
