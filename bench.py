@@ -728,14 +728,24 @@ def run_reference(args):
     n = 1
     H, M = cfg["hidden"], cfg["mlp"]
     k = [synth.keep_count(K, cfg["sparsity_percent"]) for K in (H, cfg["n_heads"] * 128, H, M)]
-    gen = torch.Generator().manual_seed(cfg["seed"])
-
-    def w(K, N):
-        return (torch.randn(K, N, generator=gen) * 0.02).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
-
     n_qkv = (cfg["n_heads"] + 2 * cfg["n_kv_heads"]) * 128
-    lw = ol.LayerWeights(w(H, n_qkv), w(cfg["n_heads"] * 128, H), w(H, M), w(H, M), w(M, H), np.ones(H), np.ones(H),
-                         k=dict(zip(("qkv", "o", "gu", "down"), k)))
+    if torch.cuda.is_available():
+        # layer 0 of the very workload the other arm decodes: the same device-side draws, copied to the host
+        L = synth.device_layer_weights(cfg["seed"], 0, H, cfg["n_heads"], cfg["n_kv_heads"], M, cfg["dtype"])
+        host = {name: L[name].cpu().numpy().view(np.uint16) for name in ("w_qkv", "w_o", "w_gu", "w_down")}
+        wg, wu = synth.split_gate_up(host["w_gu"])
+        lw = ol.LayerWeights(host["w_qkv"], host["w_o"], wg, wu, host["w_down"], np.ones(H), np.ones(H),
+                             k=dict(zip(("qkv", "o", "gu", "down"), k)))
+        weights = "layer 0 of the workload's own weights"
+    else:  # no device to draw them on: weights of the same shapes and distribution from the host generator
+        gen = torch.Generator().manual_seed(cfg["seed"])
+
+        def w(K, N):
+            return (torch.randn(K, N, generator=gen) * 0.02).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+
+        lw = ol.LayerWeights(w(H, n_qkv), w(cfg["n_heads"] * 128, H), w(H, M), w(H, M), w(M, H), np.ones(H), np.ones(H),
+                             k=dict(zip(("qkv", "o", "gu", "down"), k)))
+        weights = "host-drawn weights of the same shapes"
     ocfg = ol.Config(cfg["dtype"], H, cfg["n_heads"], cfg["n_kv_heads"], M, mode=oracle.TOPK)
     pos = cfg["past"]
     kc, vc = synth.kv_cache(cfg["seed"], 0, 1, pos + 8, cfg["n_kv_heads"], pos)
@@ -752,12 +762,16 @@ def run_reference(args):
     dt = time.perf_counter() - t0
     ms_step = dt / args.steps * 1e3
     val = 1.0 / (ms_step * 1e-3 * cfg["n_layers"] / n)
-    sample = f"each step = layer 0 of one token on the host, scaled to {cfg['n_layers']} layers"
+    sample = f"each step = layer 0 of one token on the host ({weights}), scaled to {cfg['n_layers']} layers"
     print(json.dumps({
         "impl": "reference", "metric": "decode tokens/s (batch 1)", "value": round(val, 4), "unit": "tokens/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms_step, 3),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64 (oracle)",
-        "data": "synthetic", "config": {"workload": cfg["name"], "sample": sample},
+        "data": "synthetic",
+        "config": {"workload": cfg["name"], "layers": cfg["n_layers"], "hidden": cfg["hidden"], "mlp": cfg["mlp"],
+                   "kv_past": cfg["past"], "sparsity_percent": cfg["sparsity_percent"], "select": "top-k",
+                   "accumulate": "fp64 (oracle)", "cross_layer_depth": cfg["xl_depth"], "cross_layer_mode": "bookkeeping",
+                   "sample": sample},
         "cpu_baseline": {"value": round(val, 4), "unit": "tokens/s", "cores": oracle.threads(), "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": round(val, 4), "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -1128,7 +1142,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-variants", action="store_true", help="skip the threshold / reuse variants")
     ap.add_argument("--layers", type=int, default=0, help="run only the first N layers (profiling aid)")
-    ap.add_argument("--workload", default="decode7b", choices=["decode7b", "cache70b", "swap70b"],
+    ap.add_argument("--workload", default="decode7b", choices=["decode7b", "cache70b", "swap70b", "q4"],
                     help="decode7b: the headline decode token; cache70b: host-resident weights behind the LFU cache; "
                          "swap70b: host-resident weights with cross-layer-group preloading")
     ap.add_argument("--swap-tokens", type=int, default=5, help="tokens of the swap70b workload (the first one warms up)")
@@ -1140,6 +1154,10 @@ def main():
         run_cache70b(args)
     elif args.workload == "swap70b":
         run_swap70b(args)
+    elif args.workload == "q4":  # the 4-bit sparse GEMV at the 7B operator shapes
+        import torch
+        torch.cuda.set_device(0)
+        print(json.dumps(variant_q4(torch.cuda.Stream(), measured_peaks()[0]["hbm_gbs"])))
     else:
         run_afx(args)
 
