@@ -23,8 +23,9 @@ namespace cg = cooperative_groups;
 
 constexpr int kQ4Threads = 512;
 constexpr int kQ4Warps = kQ4Threads / 32;
-constexpr int kQ4Unroll = 4;   // 16-byte loads in flight per lane
+constexpr int kQ4Unroll = 8;   // 8-byte loads in flight per lane
 constexpr int kQ4Cap = 1024;   // staged list entries per pass
+constexpr int kQ4Opl = 16;     // outputs per lane and channel: half a block of 32
 
 struct Q4Args {
     const unsigned char* Wq;
@@ -38,24 +39,38 @@ struct Q4Args {
     int32_t* status;
 };
 
-// (code - 8) for the four codes in the low nibbles of v's bytes, as two fp32 pairs.
-__device__ __forceinline__ void nibbles_to_pairs(uint32_t v, f32x2& p01, f32x2& p23) {
-    const uint32_t magic = 0x4B000000u;  // 2^23: the low mantissa byte becomes the code
-    const float bias = 8388616.0f;       // 2^23 + 8
-    const float f0 = __uint_as_float(__byte_perm(v, magic, 0x7540)) - bias;
-    const float f1 = __uint_as_float(__byte_perm(v, magic, 0x7541)) - bias;
-    const float f2 = __uint_as_float(__byte_perm(v, magic, 0x7542)) - bias;
-    const float f3 = __uint_as_float(__byte_perm(v, magic, 0x7543)) - bias;
-    p01 = pack_f32x2(f0, f1);
-    p23 = pack_f32x2(f2, f3);
+__device__ __forceinline__ uint2 ld_stream_8B(const void* p) {
+    uint2 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ f32x2 add_f32x2(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
 }
 
-// LPC lanes (blocks of 32 outputs) per channel piece: tile = LPC * 32 outputs.
+// (code - 8) for the four codes in the low nibbles of v's bytes, as two fp32 pairs: a byte
+// permute drops each code into the mantissa of 2^23 (0x4B0000qq = 2^23 + code), one two-wide
+// add takes 2^23 + 8 away again.
+__device__ __forceinline__ void nibbles_to_pairs(uint32_t v, f32x2& p01, f32x2& p23) {
+    const uint32_t magic = 0x4B000000u;
+    const f32x2 bias = pack_f32x2(-8388616.0f, -8388616.0f);
+    f32x2 a, b;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(a) : "r"(__byte_perm(v, magic, 0x7540)), "r"(__byte_perm(v, magic, 0x7541)));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(b) : "r"(__byte_perm(v, magic, 0x7542)), "r"(__byte_perm(v, magic, 0x7543)));
+    p01 = add_f32x2(a, bias);
+    p23 = add_f32x2(b, bias);
+}
+
+// A lane owns 16 outputs of a channel: bytes 8h .. 8h+7 of a block's 16 code bytes (h = 0, 1),
+// i.e. outputs 8h .. 8h+7 (low nibbles) and 16+8h .. 16+8h+7 (high nibbles) of the block.
+// LPC lanes per channel piece: tile = LPC * 16 outputs.  Two blocks of 512 threads per SM.
 template <int XDT, int LPC>
-__global__ void __launch_bounds__(kQ4Threads, 1) sparse_gemv_q4_kernel(Q4Args a) {
+__global__ void __launch_bounds__(kQ4Threads, 2) sparse_gemv_q4_kernel(Q4Args a) {
     constexpr int SUB = 32 / LPC;        // channels per warp-wide load
     constexpr int EG = kQ4Warps * SUB;   // channel groups of the block
-    constexpr int PW = LPC * 32;         // outputs of the tile
+    constexpr int PW = LPC * kQ4Opl;     // outputs of the tile
     extern __shared__ __align__(16) unsigned char q4_dyn[];
     uint32_t* s_off = reinterpret_cast<uint32_t*>(q4_dyn);          // [kQ4Cap] row offset in 16-byte units
     float* s_x = reinterpret_cast<float*>(s_off + kQ4Cap);          // [kQ4Cap]
@@ -75,16 +90,16 @@ __global__ void __launch_bounds__(kQ4Threads, 1) sparse_gemv_q4_kernel(Q4Args a)
     }
     const int c_lo = static_cast<int>(static_cast<int64_t>(rank) * cnt / S);
     const int c_hi = static_cast<int>(static_cast<int64_t>(rank + 1) * cnt / S);
-    const int blk = tile * LPC + (lane % LPC);  // this lane's block of 32 outputs
-    const bool lane_ok = blk * 32 < a.N;
+    const int half = tile * LPC + (lane % LPC);  // this lane's half block: block half >> 1, bytes 8 * (half & 1) ..
+    const bool lane_ok = half * kQ4Opl < a.N;
     const uint64_t ld16 = static_cast<uint64_t>(a.ldq >> 4);
-    const uint4* codes = reinterpret_cast<const uint4*>(a.Wq) + blk;                        // + row offset
-    const uint16_t* scales = reinterpret_cast<const uint16_t*>(a.Wq + (a.N >> 1)) + blk;    // + row offset * 8
+    const uint2* codes = reinterpret_cast<const uint2*>(a.Wq) + half;                               // + row offset * 2
+    const uint16_t* scales = reinterpret_cast<const uint16_t*>(a.Wq + (a.N >> 1)) + (half >> 1);    // + row offset * 8
     const int eg = warp * SUB + lane / LPC;
 
-    f32x2 acc[16];
+    f32x2 acc[8];  // pairs (0,1) (2,3) (4,5) (6,7) of the low nibbles, then of the high nibbles
 #pragma unroll
-    for (int i = 0; i < 16; ++i) acc[i] = pack_f32x2(0.0f, 0.0f);
+    for (int i = 0; i < 8; ++i) acc[i] = pack_f32x2(0.0f, 0.0f);
 
     for (int c0 = c_lo; c0 < c_hi; c0 += kQ4Cap) {
         int staged = min(kQ4Cap, c_hi - c0);
@@ -118,14 +133,14 @@ __global__ void __launch_bounds__(kQ4Threads, 1) sparse_gemv_q4_kernel(Q4Args a)
         }
         if (lane_ok) {
             for (int p = eg; p < staged; p += EG * kQ4Unroll) {
-                uint4 raw[kQ4Unroll];
+                uint2 raw[kQ4Unroll];
                 uint16_t sc[kQ4Unroll];
 #pragma unroll
                 for (int u = 0; u < kQ4Unroll; ++u) {
                     const int pp = p + u * EG;
                     if (pp < staged) {
                         const uint32_t off = s_off[pp];
-                        raw[u] = ld_stream_16B(codes + off);
+                        raw[u] = ld_stream_8B(codes + static_cast<size_t>(off) * 2);
                         sc[u] = __ldg(scales + static_cast<size_t>(off) * 8);
                     }
                 }
@@ -135,16 +150,16 @@ __global__ void __launch_bounds__(kQ4Threads, 1) sparse_gemv_q4_kernel(Q4Args a)
                     if (pp < staged) {
                         const float s = s_x[pp] * __half2float(__ushort_as_half(sc[u]));
                         const f32x2 s2 = pack_f32x2(s, s);
-                        const uint32_t w[4] = {raw[u].x, raw[u].y, raw[u].z, raw[u].w};
+                        const uint32_t w[2] = {raw[u].x, raw[u].y};
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {  // word q: outputs 4q..4q+3 (low nibbles), 16+4q.. (high)
+                        for (int q = 0; q < 2; ++q) {  // word q: this lane's outputs 4q..4q+3 (low nibbles), 8+4q.. (high)
                             f32x2 a01, a23;
                             nibbles_to_pairs(w[q] & 0x0F0F0F0Fu, a01, a23);
                             fma_f32x2(acc[2 * q], a01, s2);
                             fma_f32x2(acc[2 * q + 1], a23, s2);
                             nibbles_to_pairs((w[q] >> 4) & 0x0F0F0F0Fu, a01, a23);
-                            fma_f32x2(acc[8 + 2 * q], a01, s2);
-                            fma_f32x2(acc[8 + 2 * q + 1], a23, s2);
+                            fma_f32x2(acc[4 + 2 * q], a01, s2);
+                            fma_f32x2(acc[4 + 2 * q + 1], a23, s2);
                         }
                     }
                 }
@@ -152,18 +167,24 @@ __global__ void __launch_bounds__(kQ4Threads, 1) sparse_gemv_q4_kernel(Q4Args a)
         }
     }
     // ---- lane groups of a warp, warps of the block, blocks of the cluster: fixed order ----
-    float v[32];
+    float v[kQ4Opl];
 #pragma unroll
-    for (int i = 0; i < 16; ++i) unpack_f32x2(acc[i], v[2 * i], v[2 * i + 1]);
+    for (int i = 0; i < 8; ++i) unpack_f32x2(acc[i], v[2 * i], v[2 * i + 1]);
 #pragma unroll
     for (int o = LPC; o < 32; o <<= 1)
 #pragma unroll
-        for (int i = 0; i < 32; ++i) v[i] += __shfl_xor_sync(0xFFFFFFFFu, v[i], o);
+        for (int i = 0; i < kQ4Opl; ++i) v[i] += __shfl_xor_sync(0xFFFFFFFFu, v[i], o);
     __syncthreads();
+    // position of this lane's 16 values inside the tile: block (lane / 2), bytes 8h..: outputs
+    // 32 * blk + 8h + i (i < 8) and 32 * blk + 16 + 8h + i
     if (lane < LPC) {
-        float4* d4 = reinterpret_cast<float4*>(s_red + warp * PW + lane * 32);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) d4[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+        const int base = warp * PW + (lane >> 1) * 32 + (lane & 1) * 8;
+        float4* lo4 = reinterpret_cast<float4*>(s_red + base);
+        float4* hi4 = reinterpret_cast<float4*>(s_red + base + 16);
+        lo4[0] = make_float4(v[0], v[1], v[2], v[3]);
+        lo4[1] = make_float4(v[4], v[5], v[6], v[7]);
+        hi4[0] = make_float4(v[8], v[9], v[10], v[11]);
+        hi4[1] = make_float4(v[12], v[13], v[14], v[15]);
     }
     __syncthreads();
     float* part = s_red + kQ4Warps * PW;  // this block's sums, read by the cluster
@@ -186,19 +207,19 @@ __global__ void __launch_bounds__(kQ4Threads, 1) sparse_gemv_q4_kernel(Q4Args a)
 }
 
 static size_t q4_dyn_smem(int lpc) {
-    return static_cast<size_t>(kQ4Cap) * 8 + static_cast<size_t>(kQ4Warps + 1) * lpc * 32 * 4;
+    return static_cast<size_t>(kQ4Cap) * 8 + static_cast<size_t>(kQ4Warps + 1) * lpc * kQ4Opl * 4;
 }
 
 template <int XDT>
 static afx_status launch_q4(const Q4Args& a, cudaStream_t st) {
     const void* kerns[3] = {reinterpret_cast<const void*>(sparse_gemv_q4_kernel<XDT, 32>),
-                            reinterpret_cast<const void*>(sparse_gemv_q4_kernel<XDT, 8>),
-                            reinterpret_cast<const void*>(sparse_gemv_q4_kernel<XDT, 4>)};
-    const int lpcs[3] = {32, 8, 4};
+                            reinterpret_cast<const void*>(sparse_gemv_q4_kernel<XDT, 16>),
+                            reinterpret_cast<const void*>(sparse_gemv_q4_kernel<XDT, 8>)};
+    const int lpcs[3] = {32, 16, 8};
     // the widest tile and largest cluster that keep every cluster resident at once, most blocks wins
     int best = 2, best_S = 1, best_blocks = -1;
     for (int i = 0; i < 3; ++i) {
-        const int tiles = (a.N + lpcs[i] * 32 - 1) / (lpcs[i] * 32);
+        const int tiles = (a.N + lpcs[i] * kQ4Opl - 1) / (lpcs[i] * kQ4Opl);
         const size_t dyn = q4_dyn_smem(lpcs[i]);
         for (int S = kMaxCluster; S >= 1; --S) {
             const int margin = (tiles + 15) / 16 < 2 ? 2 : (tiles + 15) / 16;
@@ -213,13 +234,13 @@ static afx_status launch_q4(const Q4Args& a, cudaStream_t st) {
         }
     }
     const int lpc = lpcs[best];
-    const int tiles = (a.N + lpc * 32 - 1) / (lpc * 32);
+    const int tiles = (a.N + lpc * kQ4Opl - 1) / (lpc * kQ4Opl);
     if (tiles > 65535) return AFX_ERR_CAPACITY;
     const size_t dyn = q4_dyn_smem(lpc);
     switch (lpc) {
         case 32: return launch_clustered(sparse_gemv_q4_kernel<XDT, 32>, best_S, tiles, dyn, a, st, kQ4Threads);
-        case 8: return launch_clustered(sparse_gemv_q4_kernel<XDT, 8>, best_S, tiles, dyn, a, st, kQ4Threads);
-        default: return launch_clustered(sparse_gemv_q4_kernel<XDT, 4>, best_S, tiles, dyn, a, st, kQ4Threads);
+        case 16: return launch_clustered(sparse_gemv_q4_kernel<XDT, 16>, best_S, tiles, dyn, a, st, kQ4Threads);
+        default: return launch_clustered(sparse_gemv_q4_kernel<XDT, 8>, best_S, tiles, dyn, a, st, kQ4Threads);
     }
 }
 
