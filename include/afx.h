@@ -422,7 +422,7 @@ afx_status afx_swap_pack_host(const void* const* per_layer, int n_layers, int gr
 size_t afx_swap_device_bytes(const afx_swap_desc* desc);
 
 /* Resolves the device view of host_base (AFX_ERR_INVALID_ARG when it is not page-locked),
- * allocates the tables (cudaMalloc, about 12 bytes per channel), creates the events and, if
+ * allocates the tables (cudaMalloc, about 20 bytes per channel), creates the events and, if
  * none was given, the loader stream.  afx_swap_destroy releases them. */
 afx_status afx_swap_create(const afx_swap_desc* desc, afx_swap** out);
 afx_status afx_swap_destroy(afx_swap* swap);
@@ -430,8 +430,9 @@ afx_status afx_swap_destroy(afx_swap* swap);
 /*
  * PL: preload group `group_index` from the predicted list idxP[0 .. *cntP) (DEVICE, ascending, as
  * afx_select_active or a layer step writes it).  Enqueued on the loader stream behind everything
- * enqueued on compute_stream so far (the list must have been produced there); predicted
- * channel c goes to row c of every layer of the group.  copy_blocks: thread blocks of the copy
+ * enqueued on compute_stream so far (the list must have been produced there; idxP must hold K
+ * readable entries: the call first takes its own copy on compute_stream, so the caller may
+ * overwrite the list afterwards); predicted channel c goes to row c of every layer of the group.  copy_blocks: thread blocks of the copy
  * kernel (0 = 32; it reads host memory over PCIe and needs few).  Call it only after the
  * compute stream has been given all work of group_index - 2, whose buffer it overwrites.
  */
@@ -567,6 +568,27 @@ size_t afx_moe_workspace_bytes(const afx_moe_desc* desc);
  */
 afx_status afx_moe_block(const afx_moe_desc* desc, const void* x, float* y, int accumulate, void* workspace,
                          size_t workspace_bytes, void* stream);
+
+/*
+ * afx_layer_step for a layer some of whose operators do not live in device memory: per
+ * operator input (AFX_OP_*) either an LFU cache (afx_cache: THIS layer's operator tensor) or a
+ * swapping object (afx_swap: the operator type of all layers).  Such an operator runs as the
+ * paper's pipeline stages one after the other on `stream` -- T: input stage + selection (the
+ * side outputs of the fused kernel: normed input, active list, cross-layer bookkeeping), L:
+ * afx_cache_fetch / afx_swap_acquire, C: the sparse GEMV through the slot list with the
+ * operator's epilogue -- while operators with neither handle run fused on the resident weights
+ * of the layer descriptor.  slot[op]: DEVICE int32[K_op] scratch for the slot list.  Preloads
+ * (afx_swap_preload from the state's AFX_BUF_IDX list) are the caller's to request between layer
+ * steps.  AFX_XL_REUSE models are not supported.  q|k|v, gate|up (interleaved) and the
+ * other operators use the layouts of afx_layer_desc in their host images.
+ */
+typedef struct {
+    afx_cache* cache[4]; /* per AFX_OP_*: or NULL */
+    afx_swap* swap[4];   /* per AFX_OP_*: or NULL (not both)                                      */
+    int32_t* slot[4];    /* DEVICE int32[K_op] where a handle is given                            */
+} afx_hosted_ops;
+afx_status afx_layer_step_hosted(afx_model* model, int layer, afx_state* state, int pos, const afx_hosted_ops* ops,
+                                 int32_t* dev_status, void* stream);
 
 /*
  * The MLP block without any allocation (the paper has no counterpart: this entry point exists

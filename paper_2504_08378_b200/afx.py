@@ -108,6 +108,11 @@ class MoeDesc(ctypes.Structure):
                 ("w_down_table", c_void_p)]
 
 
+class HostedOps(ctypes.Structure):
+    """afx_hosted_ops"""
+    _fields_ = [("cache", c_void_p * 4), ("swap", c_void_p * 4), ("slot", c_void_p * 4)]
+
+
 class AfxError(RuntimeError):
     def __init__(self, fn: str, status: int):
         self.status = status
@@ -174,6 +179,7 @@ def lib() -> ctypes.CDLL:
         L.afx_q4_row_bytes.argtypes = [c_int]
         L.afx_sparse_gemv_q4.argtypes = [c_void_p, c_int, c_int, c_int64, c_void_p, c_int, c_void_p, c_void_p, c_void_p,
                                          c_int, c_void_p, c_void_p]
+        L.afx_layer_step_hosted.argtypes = [c_void_p, c_int, c_void_p, c_int, ctypes.POINTER(HostedOps), c_void_p, c_void_p]
         L.afx_mlp_block_noalloc.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_void_p, c_int, c_int, c_int,
                                             c_float, c_int, c_float, c_void_p, c_void_p]
         _lib = L
@@ -423,3 +429,8 @@ def afx_sparse_gemv_q4(Wq, K: int, N: int, ldq_bytes: int, x, x_dtype, idx, coun
     _check("afx_sparse_gemv_q4",
            lib().afx_sparse_gemv_q4(_ptr(Wq), int(K), int(N), int(ldq_bytes), _ptr(x), _dt(x_dtype), _ptr(idx), _ptr(count),
                                     _ptr(y), int(accumulate), _ptr(dev_status), _stream(stream)))
+
+
+def afx_layer_step_hosted(model: int, layer: int, state: int, pos: int, ops: HostedOps, stream=None, dev_status=None):
+    _check("afx_layer_step_hosted", lib().afx_layer_step_hosted(model, int(layer), state, int(pos), ctypes.byref(ops),
+                                                                _ptr(dev_status), _stream(stream)))

@@ -246,6 +246,10 @@ struct afx_cache {
     void* arena;           // one cudaMalloc holding every table
 };
 
+namespace afx {
+HostedRows cache_rows(const afx_cache* cache) { return {cache->d.slots, cache->d.ldw, cache->d.K, cache->d.N}; }
+}  // namespace afx
+
 extern "C" afx_status afx_cache_create(const afx_cache_desc* desc, afx_cache** out) {
     using namespace afx;
     if (desc == nullptr || out == nullptr) return AFX_ERR_INVALID_ARG;

@@ -56,6 +56,10 @@ static afx_status launch_gemv(const GemvListArgs& a, cudaStream_t st) {
     return launch_gemv_t<DT, 8>(a, st);
 }
 
+afx_status launch_list_gemv(int dtype, const GemvListArgs& a, cudaStream_t st) {
+    return dtype == AFX_F16 ? launch_gemv<AFX_F16>(a, st) : launch_gemv<AFX_BF16>(a, st);
+}
+
 }  // namespace afx
 
 #ifdef AFX_EXPERIMENT
@@ -100,11 +104,11 @@ extern "C" afx_status afx_sparse_gemv(const void* Wt, int dtype, int K, int N, i
     a.count = count;
     a.slot = slot;
     a.accumulate = accumulate ? 1 : 0;
+    a.silu = 0;
     a.ep.y = y;
     a.ep.out_bits = nullptr;
     a.ep.N = N;
     a.ep.scale = nullptr;
     a.status = dev_status;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    return dtype == AFX_F16 ? launch_gemv<AFX_F16>(a, st) : launch_gemv<AFX_BF16>(a, st);
+    return launch_list_gemv(dtype, a, static_cast<cudaStream_t>(stream));
 }

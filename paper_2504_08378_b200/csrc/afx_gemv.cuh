@@ -235,10 +235,14 @@ struct GemvListArgs {
     const int32_t* idx;
     const int32_t* count;
     const int32_t* slot;
-    int accumulate;
+    int accumulate;   // 0: y = sum, 1: y += sum
+    int silu;         // 1: gate|up columns, out_bits = round(silu(gate) * up) instead of y
     EpilogueArgs ep;
     int32_t* status;  // device status word or NULL
 };
+
+// afx_sparse_gemv's launcher (afx_gemv.cu), also used by the layer step over host-resident weights.
+afx_status launch_list_gemv(int dtype, const GemvListArgs& a, cudaStream_t st);
 
 // grid = (S, tiles), cluster = (S, 1, 1).
 template <int DT, int TMAX, int PW, int CAP>
@@ -316,7 +320,9 @@ __device__ __forceinline__ void gemv_list_block(const GemvListArgs& a, GemvSmem<
         }
         if (lane_ok) gemv_stream<DT, TMAX, PW, CAP, true>(wbase16, T, sm, staged, acc);
     }
-    if (a.accumulate)
+    if (a.silu)
+        gemv_finish_tile<DT, TMAX, PW, CAP, EP_SILU>(acc, T, tile, sm, recv, a.ep);
+    else if (a.accumulate)
         gemv_finish_tile<DT, TMAX, PW, CAP, EP_ACCUM>(acc, T, tile, sm, recv, a.ep);
     else
         gemv_finish_tile<DT, TMAX, PW, CAP, EP_STORE>(acc, T, tile, sm, recv, a.ep);

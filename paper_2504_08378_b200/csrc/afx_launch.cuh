@@ -77,6 +77,15 @@ inline int max_active_clusters(const void* kern, int S, size_t dyn_smem, int thr
     return n;
 }
 
+// Where the device rows of a host-resident operator live (for the layer step over such operators).
+struct HostedRows {
+    const void* rows;
+    int64_t ldw;
+    int K, N;
+};
+HostedRows cache_rows(const afx_cache* cache);  // afx_cache.cu
+HostedRows swap_rows(const afx_swap* swap);     // afx_swap.cu (rows = NULL: afx_swap_acquire returns them per layer)
+
 struct GemvShapeChoice {
     int pw;     // tile width: 256, 128 or 64 outputs
     int S;      // blocks per cluster (= per tile)

@@ -428,6 +428,117 @@ extern "C" afx_status afx_layer_kernel(afx_model* m, int layer, afx_state* s, in
     return launch_layer_kernel(m, layer, s, pos, which, static_cast<cudaStream_t>(stream));
 }
 
+namespace afx {
+
+// Input stage + selection of one operator WITHOUT its GEMV: one block that writes what a fused
+// launch's side-output block writes (normed input, active list, count, cross-layer bookkeeping).
+template <int IN>
+static afx_status launch_select_only(int dtype, const FusedArgs& a, cudaStream_t st) {
+    FusedArgs b = a;
+    b.side_cluster = 1;
+    b.N = 8;  // no column tile is streamed: the grid holds the side-output cluster only
+    const size_t dyn = fused_dyn_smem(IN, a.K, a.T);
+    auto go = [&](auto kern) { return launch_clustered(kern, 1, 1, dyn, b, st); };
+    if (dtype == AFX_F16) {
+        if (a.T <= 1) return go(fused_op_kernel<AFX_F16, 1, 64, IN, EP_STORE>);
+        if (a.T <= 4) return go(fused_op_kernel<AFX_F16, 4, 64, IN, EP_STORE>);
+        return go(fused_op_kernel<AFX_F16, 8, 64, IN, EP_STORE>);
+    }
+    if (a.T <= 1) return go(fused_op_kernel<AFX_BF16, 1, 64, IN, EP_STORE>);
+    if (a.T <= 4) return go(fused_op_kernel<AFX_BF16, 4, 64, IN, EP_STORE>);
+    return go(fused_op_kernel<AFX_BF16, 8, 64, IN, EP_STORE>);
+}
+
+}  // namespace afx
+
+extern "C" afx_status afx_layer_step_hosted(afx_model* m, int layer, afx_state* s, int pos, const afx_hosted_ops* ops,
+                                            int32_t* dev_status, void* stream) {
+    using namespace afx;
+    afx_status rc = check_step(m, layer, s);
+    if (rc != AFX_OK) return rc;
+    if (ops == nullptr || pos < 0 || pos >= m->d.max_seq) return AFX_ERR_INVALID_ARG;
+    if (m->d.xl_mode == AFX_XL_REUSE) return AFX_ERR_UNSUPPORTED;  // a hosted operator always selects for itself
+    const afx_model_desc& d = m->d;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int N_op[4] = {m->n_qkv, d.hidden, 2 * d.mlp, d.hidden};
+    for (int op = 0; op < 4; ++op) {
+        const bool hosted = ops->cache[op] != nullptr || ops->swap[op] != nullptr;
+        if (ops->cache[op] != nullptr && ops->swap[op] != nullptr) return AFX_ERR_INVALID_ARG;
+        if (hosted && (ops->slot[op] == nullptr || (reinterpret_cast<uintptr_t>(ops->slot[op]) & 3u) != 0))
+            return ops->slot[op] == nullptr ? AFX_ERR_INVALID_ARG : AFX_ERR_ALIGNMENT;
+        if (hosted) {
+            const HostedRows r = ops->cache[op] != nullptr ? cache_rows(ops->cache[op]) : swap_rows(ops->swap[op]);
+            if (r.K != m->K_op[op] || r.N != N_op[op]) return AFX_ERR_INVALID_ARG;
+        }
+    }
+    float* h = reinterpret_cast<float*>(s->blob + s->off_h);
+    float* qkv = reinterpret_cast<float*>(s->blob + s->off_qkv);
+    uint16_t* attn = reinterpret_cast<uint16_t*>(s->blob + s->off_attn);
+    uint16_t* hm = reinterpret_cast<uint16_t*>(s->blob + s->off_hm);
+    int32_t* stats = reinterpret_cast<int32_t*>(s->blob + s->off_stats);
+    const afx_layer_desc& L = m->layers[layer];
+    const int which_of[4] = {AFX_STEP_QKV, AFX_STEP_O, AFX_STEP_GU, AFX_STEP_DOWN};
+    for (int op = 0; op < 4; ++op) {
+        if (op == AFX_OP_O && (rc = launch_layer_kernel(m, layer, s, pos, AFX_STEP_ATTN, st)) != AFX_OK) return rc;
+        if (ops->cache[op] == nullptr && ops->swap[op] == nullptr) {  // resident weights: the fused kernel
+            if ((rc = launch_layer_kernel(m, layer, s, pos, which_of[op], st)) != AFX_OK) return rc;
+            continue;
+        }
+        // 1. input stage + selection
+        FusedArgs a = {};
+        a.T = s->T;
+        a.eps = d.rms_eps;
+        a.K = m->K_op[op];
+        a.ldw = N_op[op];
+        const uint16_t* x16 = nullptr;  // the operator's 16-bit input
+        const bool norm = op == AFX_OP_QKV || op == AFX_OP_GU;
+        if (norm) {
+            a.h = h;
+            a.gain = op == AFX_OP_QKV ? L.g_attn : L.g_mlp;
+            a.xnorm_out = reinterpret_cast<uint16_t*>(s->blob + s->off_xnorm[op == AFX_OP_QKV ? 0 : 1]);
+            x16 = a.xnorm_out;
+        } else {
+            a.x = op == AFX_OP_O ? attn : hm;
+            x16 = a.x;
+        }
+        plan_selection(m, s, layer, op, true, &a);
+        rc = norm ? launch_select_only<IN_NORM>(d.dtype, a, st) : launch_select_only<IN_X>(d.dtype, a, st);
+        if (rc != AFX_OK) return rc;
+        const int32_t* idx = a.idx_out;
+        const int32_t* count = stats + (static_cast<size_t>(layer) * 4 + op) * 4;
+        // 2. where the active columns are (fetching what is missing)
+        GemvListArgs g = {};
+        if (ops->cache[op] != nullptr) {
+            const HostedRows r = cache_rows(ops->cache[op]);
+            g.Wt = static_cast<const uint16_t*>(r.rows);
+            g.ldw = r.ldw;
+            rc = afx_cache_fetch(ops->cache[op], idx, count, ops->slot[op], nullptr, dev_status, stream);
+        } else {
+            const void* rows = nullptr;
+            g.ldw = swap_rows(ops->swap[op]).ldw;
+            rc = afx_swap_acquire(ops->swap[op], layer, idx, count, ops->slot[op], nullptr, dev_status, stream, &rows);
+            g.Wt = static_cast<const uint16_t*>(rows);
+        }
+        if (rc != AFX_OK) return rc;
+        // 3. the operator on the fetched rows
+        g.K = m->K_op[op];
+        g.N = N_op[op];
+        g.T = s->T;
+        g.x = x16;
+        g.idx = idx;
+        g.count = count;
+        g.slot = ops->slot[op];
+        g.status = dev_status;
+        switch (op) {
+            case AFX_OP_QKV: g.ep = {qkv, nullptr, N_op[op], nullptr}; break;
+            case AFX_OP_GU: g.silu = 1; g.ep = {nullptr, hm, N_op[op], nullptr}; break;
+            default: g.accumulate = 1; g.ep = {h, nullptr, N_op[op], nullptr}; break;
+        }
+        if ((rc = launch_list_gemv(d.dtype, g, st)) != AFX_OK) return rc;
+    }
+    return AFX_OK;
+}
+
 extern "C" afx_status afx_mlp_block(afx_model* m, int layer, afx_state* s, const void* x, float* y,
                                     void* stream) {
     using namespace afx;

@@ -30,6 +30,7 @@ struct SwapDev {
     int32_t* n_pred;          // [2]: channels preloaded into the buffer
     int32_t* fetch_ch;        // [K] on-demand channels of the last acquire
     int32_t* n_fetch;         // [1]
+    int32_t* pred_list;       // [2][K + 1]: the object's own copy of a predicted list (count last)
 };
 
 __host__ __device__ inline int64_t swap_offset16(int L, int d, int K, int64_t ldw16, int layer, int channel) {
@@ -183,6 +184,10 @@ struct afx_swap {
     int n_groups = 0;
 };
 
+namespace afx {
+HostedRows swap_rows(const afx_swap* swap) { return {nullptr, swap->d.ldw, swap->d.K, swap->d.N}; }
+}  // namespace afx
+
 extern "C" size_t afx_swap_host_offset(int n_layers, int group, int K, int64_t ldw, int layer, int channel) {
     if (n_layers < 1 || group < 1 || K < 1 || ldw < 1 || layer < 0 || layer >= n_layers || channel < 0 || channel >= K)
         return static_cast<size_t>(-1);
@@ -231,7 +236,8 @@ extern "C" afx_status afx_swap_create(const afx_swap_desc* desc, afx_swap** out)
     s->n_groups = (d.n_layers + d.group - 1) / d.group;
     const size_t K = static_cast<size_t>(d.K);
     auto up = [](size_t b) { return (b + 255) / 256 * 256; };
-    const size_t o_pred = 0, o_np = o_pred + up(2 * K * 4), o_fch = o_np + 256, o_nf = o_fch + up(K * 4), total = o_nf + 256;
+    const size_t o_pred = 0, o_np = o_pred + up(2 * K * 4), o_fch = o_np + 256, o_nf = o_fch + up(K * 4),
+                 o_pl = o_nf + 256, total = o_pl + up(2 * (K + 1) * 4);
     char* arena = nullptr;
     bool ok = cudaMalloc(reinterpret_cast<void**>(&arena), total) == cudaSuccess;
     ok = ok && cudaMemset(arena, 0xFF, up(2 * K * 4)) == cudaSuccess && cudaMemset(arena + o_np, 0, total - o_np) == cudaSuccess;
@@ -265,6 +271,7 @@ extern "C" afx_status afx_swap_create(const afx_swap_desc* desc, afx_swap** out)
     v.n_pred = reinterpret_cast<int32_t*>(arena + o_np);
     v.fetch_ch = reinterpret_cast<int32_t*>(arena + o_fch);
     v.n_fetch = reinterpret_cast<int32_t*>(arena + o_nf);
+    v.pred_list = reinterpret_cast<int32_t*>(arena + o_pl);
     *out = s;
     return AFX_OK;
 }
@@ -292,12 +299,18 @@ extern "C" afx_status afx_swap_preload(afx_swap* s, int group_index, const int32
     const int b = group_index & 1;
     cudaStream_t cs = static_cast<cudaStream_t>(compute_stream);
     const int blocks = copy_blocks > 0 ? copy_blocks : 32;
+    // The caller's list may be overwritten by the next layer while the loader still reads it:
+    // take a copy on the compute stream first.
+    int32_t* own = s->dev.pred_list + static_cast<size_t>(b) * (s->dev.K + 1);
+    if (cudaMemcpyAsync(own, idxP, static_cast<size_t>(s->dev.K) * 4, cudaMemcpyDeviceToDevice, cs) != cudaSuccess ||
+        cudaMemcpyAsync(own + s->dev.K, cntP, 4, cudaMemcpyDeviceToDevice, cs) != cudaSuccess)
+        return AFX_ERR_CUDA;
     // request: the list exists, and everything that still reads this buffer has been enqueued
     if (cudaEventRecord(s->ev_req[b], cs) != cudaSuccess || cudaStreamWaitEvent(s->loader, s->ev_req[b], 0) != cudaSuccess)
         return AFX_ERR_CUDA;
     swap_clear_kernel<<<8, 256, 0, s->loader>>>(s->dev.pred_slot + static_cast<size_t>(b) * s->dev.K, s->dev.K,
                                                  s->dev.n_pred + b);
-    swap_preload_kernel<<<blocks, kSwapCopyThreads, 0, s->loader>>>(s->dev, group_index, b, idxP, cntP, dev_status);
+    swap_preload_kernel<<<blocks, kSwapCopyThreads, 0, s->loader>>>(s->dev, group_index, b, own, own + s->dev.K, dev_status);
     if (cudaGetLastError() != cudaSuccess) return AFX_ERR_CUDA;
     // complete
     if (cudaEventRecord(s->ev_done[b], s->loader) != cudaSuccess) return AFX_ERR_CUDA;
