@@ -4,15 +4,15 @@
 //
 // A channel's row is [N/2 bytes of 4-bit codes][N/32 fp16 scales]; a block of 32 outputs is 16
 // bytes of codes and one scale: byte m = code of output m (low 4 bits) and of output 16 + m
-// (high 4 bits); value = (code - 8) * scale.  One lane owns one block of one channel per load:
-// a 16-byte read of the codes plus the block's scale, x * scale once, then 32 multiply-adds with
-// the codes turned into fp32 by a byte permute into the mantissa of 2^23 (0x4B0000qq = 2^23 + q)
-// and one subtraction of 2^23 + 8 -- two-wide adds and fused multiply-adds.  The tile of a
-// cluster is LPC blocks (LPC * 32 outputs) wide; the S blocks of the cluster split the active
-// list and meet through distributed shared memory in rank order; sums are fp32 in a fixed
-// order.  3.5x fewer bytes per weight than the 16-bit kernels, but about 5 executed
-// instructions per weight: this kernel is bound by instruction issue (one 512-thread block of
-// 120+ registers per SM), not by HBM.
+// (high 4 bits); value = (code - 8) * scale.  One lane owns HALF a block of one channel per
+// load: an 8-byte read of the codes plus the block's scale, x * scale once, then 16
+// multiply-adds with the codes turned into fp32 by a byte permute into the mantissa of 2^23
+// (0x4B0000qq = 2^23 + q) and a subtraction of 2^23 + 8 -- two-wide adds and fused
+// multiply-adds.  The tile of a cluster is LPC half blocks (LPC * 16 outputs) wide; the S blocks
+// of the cluster split the active list and meet through distributed shared memory in rank
+// order; sums are fp32 in a fixed order.  3.5x fewer bytes per weight than the 16-bit kernels,
+// but 5-6 executed instructions per weight: this kernel is bound by instruction issue, not by
+// HBM (64 registers, two 512-thread blocks per SM).
 #include <cooperative_groups.h>
 
 #include "afx_launch.cuh"
