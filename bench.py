@@ -1059,7 +1059,7 @@ def variant_q4(st, peak):
     import numpy as np
     import torch
     from paper_2504_08378_b200 import afx, synth
-    out = {"note": "about 2.3 instructions per weight: bound by instruction issue before HBM"}
+    out = {"note": "5-6 executed instructions per weight (ncu): bound by instruction issue, not by HBM"}
     gen = torch.Generator(device="cuda")
     gen.manual_seed(77)
     for name, K, N in (("gate_up", 4096, 22016), ("qkv", 4096, 12288), ("down", 11008, 4096), ("o", 4096, 4096)):
