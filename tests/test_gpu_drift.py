@@ -12,8 +12,8 @@ What is gated:
   2. where the two runs' inputs of an operator still agree to within 2 key steps around the
      boundary, every channel that is in exactly one of (GPU set, oracle set) has a magnitude key
      within 2 steps of the k-th key on both sides: a rounding case at the boundary.
-What is reported (printed, and written to gpurun_out/drift_7b.json when that directory
-exists): per layer and operator the number of such channels, the Jaccard index of the two sets,
+What is reported (printed, and written to $AFX_REPORT_DIR/drift_7b.json when that variable
+names a directory): per layer and operator the number of such channels, the Jaccard index of the two sets,
 the key drift of the inputs near the boundary, and the hidden-state error; the first layer
 with a difference; the final hidden-state error.
 """
@@ -106,8 +106,8 @@ def test_free_running_7b_token_flips_only_at_topk_boundaries():
     print(json.dumps({kk: v for kk, v in report.items() if kk != "layers"}))
     for r in report["layers"]:
         print(r)
-    out_dir = os.path.join(ROOT, "gpurun_out")
-    if os.path.isdir(out_dir):
+    out_dir = os.environ.get("AFX_REPORT_DIR", "")
+    if out_dir and os.path.isdir(out_dir):
         with open(os.path.join(out_dir, "drift_7b.json"), "w") as f:
             json.dump(report, f)
     assert report["unexplained"] == 0
