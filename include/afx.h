@@ -259,6 +259,8 @@ afx_status afx_state_destroy(afx_state* state);
                              /*                       of the last one-token top-k selection (0  */
                              /*                       before the first; the next token's search */
                              /*                       starts there, any value gives the same set) */
+#define AFX_BUF_HINTS 8      /* int32 [n_layers][4][AFX_MAX_T] the same search hints per token when T > 1: */
+                             /*                       0x10000 | k-th key of token t's last selection   */
 afx_status afx_state_buffer(const afx_state* state, int which, int op, void** ptr, size_t* bytes);
 
 /*

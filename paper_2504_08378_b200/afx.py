@@ -15,7 +15,7 @@ from . import build as _build
 F16, BF16 = 0, 1
 OP_QKV, OP_O, OP_GU, OP_DOWN = 0, 1, 2, 3
 XL_OFF, XL_BOOKKEEP, XL_REUSE = 0, 1, 2
-BUF_H, BUF_QKV, BUF_ATTN, BUF_HM, BUF_XNORM, BUF_IDX, BUF_MISS, BUF_STATS = range(8)
+BUF_H, BUF_QKV, BUF_ATTN, BUF_HM, BUF_XNORM, BUF_IDX, BUF_MISS, BUF_STATS, BUF_HINTS = range(9)
 STEP_QKV, STEP_ATTN, STEP_O, STEP_GU, STEP_DOWN = range(5)
 MODE_TOPK, MODE_THRESHOLD = 0, 1
 MAX_T = 8

@@ -43,6 +43,8 @@ struct FusedArgs {
     // ---- top-k search hint (may be NULL): 0x10000 | k-th key of this operator's last top-k
     // selection with T == 1; read before the selection, rewritten after it by block (0,0) ----
     int32_t* kth_slot;
+    // ---- the same for several tokens (T > 1; may be NULL): T consecutive slots, one per token ----
+    int32_t* kth_multi;
     // ---- set by the launcher: 1 if the grid has one more cluster than column tiles; its block 0
     // repeats input stage and selection only to write the side outputs, off the path of the
     // clusters that stream (its other blocks leave at once) ----
@@ -118,6 +120,15 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
     if (topk && T == 1 && a.kth_slot != nullptr) {
         const uint32_t v = static_cast<uint32_t>(__ldcg(a.kth_slot));
         if (v & 0x10000u) hint = v & 0x7FFFu;
+    }
+    uint32_t hint_t[TMAX];  // several tokens: one hint each
+#pragma unroll
+    for (int t = 0; t < TMAX; ++t) {
+        hint_t[t] = kNoKeyHint;
+        if (TMAX > 1 && topk && T > 1 && t < T && a.kth_multi != nullptr) {
+            const uint32_t v = static_cast<uint32_t>(__ldcg(a.kth_multi + t));
+            if (v & 0x10000u) hint_t[t] = v & 0x7FFFu;
+        }
     }
     // likewise the predicted set this selection is compared with: the same operator of the
     // predictor layer wrote it, at least one layer (five grids) ago (byte v = the flags of the
@@ -233,8 +244,14 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
                 first_staged = true;
                 if (scribe && tid == 0 && a.kth_slot != nullptr) *a.kth_slot = 0x10000 | sel->res[0];
             } else {
+                uint32_t thr_t = 0;
+                uint32_t h_t = kNoKeyHint;
+#pragma unroll
+                for (int u = 0; u < TMAX; ++u)
+                    if (u == t) h_t = hint_t[u];
                 fl |= block_token_flags<DT, kGemvThreads>(xt, K, a.mode, a.k, a.tau, hist, t == 0, sel, T == 1,
-                                                          pos0, cnt);
+                                                          pos0, cnt, NoEmit(), 0, 0x7FFFFFFF, h_t, nullptr, &thr_t);
+                if (scribe && tid == 0 && topk && T > 1 && a.kth_multi != nullptr) a.kth_multi[t] = 0x10000 | thr_t;
             }
         }
         if (T > 1) pos0 = block_prefix(__popcll(fl), sel->wtot[2], cnt);

@@ -50,7 +50,8 @@ static afx_status launch_fused_t(const FusedArgs& a, cudaStream_t st) {
     // side outputs, if any, come from one more cluster than there are column tiles
     FusedArgs b = a;
     b.side_cluster = (a.idx_out != nullptr || a.count_out != nullptr || a.bitmap_out != nullptr ||
-                      a.xnorm_out != nullptr || a.bitmap_pred != nullptr || a.kth_slot != nullptr)
+                      a.xnorm_out != nullptr || a.bitmap_pred != nullptr || a.kth_slot != nullptr ||
+                      (a.kth_multi != nullptr && a.T > 1))
                          ? 1 : 0;
     const GemvShapeChoice c = choose_gemv_shape(a.N, kerns, dyn, b.side_cluster);
     if (c.tiles + b.side_cluster > 65535) return AFX_ERR_CAPACITY;
@@ -115,8 +116,8 @@ struct afx_state {
     int T;
     char* blob;
     size_t bytes;
-    size_t off_h, off_qkv, off_attn, off_hm, off_xnorm[2], off_idx[4], off_miss[4], off_pred[4][2], off_stats;
-    size_t sz_h, sz_qkv, sz_attn, sz_hm, sz_xnorm, sz_idx[4], sz_pred[4], sz_stats;
+    size_t off_h, off_qkv, off_attn, off_hm, off_xnorm[2], off_idx[4], off_miss[4], off_pred[4][2], off_stats, off_hints;
+    size_t sz_h, sz_qkv, sz_attn, sz_hm, sz_xnorm, sz_idx[4], sz_pred[4], sz_stats, sz_hints;
 };
 
 static void state_layout(const afx_model* m, int T, afx_state* s) {
@@ -149,6 +150,8 @@ static void state_layout(const afx_model* m, int T, afx_state* s) {
     }
     s->sz_stats = static_cast<size_t>(d.n_layers) * 4 * 4 * 4;
     s->off_stats = take(s->sz_stats);
+    s->sz_hints = static_cast<size_t>(d.n_layers) * 4 * AFX_MAX_T * 4;
+    s->off_hints = take(s->sz_hints);
     s->bytes = o;
 }
 
@@ -274,6 +277,7 @@ extern "C" afx_status afx_state_buffer(const afx_state* s, int which, int op, vo
             if (op < 0 || op > 3) return AFX_ERR_INVALID_ARG;
             off = s->off_miss[op]; sz = s->sz_idx[op]; break;
         case AFX_BUF_STATS: off = s->off_stats; sz = s->sz_stats; break;
+        case AFX_BUF_HINTS: off = s->off_hints; sz = s->sz_hints; break;
         default: return AFX_ERR_INVALID_ARG;
     }
     *ptr = s->blob + off;
@@ -303,6 +307,7 @@ static void plan_selection(const afx_model* m, const afx_state* s, int layer, in
     a->miss_count = nullptr;
     a->hit_count = nullptr;
     a->kth_slot = my_stats + 3;
+    a->kth_multi = reinterpret_cast<int32_t*>(s->blob + s->off_hints) + (static_cast<size_t>(layer) * 4 + op) * AFX_MAX_T;
     const int depth = d.xl_depth;
     if (!cross_layer || depth <= 0 || d.xl_mode == AFX_XL_OFF) return;
     const bool predictor = (layer % depth) == 0;

@@ -341,9 +341,9 @@ __device__ __forceinline__ bool block_kth_key_near(const uint16_t* xs, int K, in
 // returns the list position of the thread's first active channel in `pos0` and the length
 // of the list in `cnt`, from the same scan that orders the tie-break, and calls
 // emit(channel, list position, 16-bit pattern) for the thread's active channels (only for a
-// thread that can own a position in [emit_lo, emit_hi)).  `hint` (top-k,
-// `single` only; kNoKeyHint = none) is a guess of the k-th key that shortens the search and
-// never changes the result.  `xchg` (top-k emits; may be NULL) is ceil(K/8) words of shared
+// thread that can own a position in [emit_lo, emit_hi)).  `hint` (top-k; kNoKeyHint = none) is
+// a guess of the k-th key that shortens the search and never changes the result; `thr_out`
+// (top-k with 0 < k < K) receives the k-th key found, in every thread.  `xchg` (top-k emits; may be NULL) is ceil(K/8) words of shared
 // memory apart from the histogram's first KeyWindow bins and from whatever emit writes.
 // After a top-k selection with 0 < k < K, s->res[0] holds the k-th
 // key until the next selection.
@@ -370,7 +370,8 @@ __device__ __forceinline__ unsigned long long block_token_flags(const uint16_t* 
                                                                 int& cnt, Emit emit = Emit(), int emit_lo = 0,
                                                                 int emit_hi = 0x7FFFFFFF,
                                                                 uint32_t hint = kNoKeyHint,
-                                                                uint32_t* xchg = nullptr) {
+                                                                uint32_t* xchg = nullptr,
+                                                                uint32_t* thr_out = nullptr) {
     int c_lo, c_hi;
     thread_chunk_range(K, c_lo, c_hi);
     unsigned long long fl = 0ull;
@@ -407,13 +408,15 @@ __device__ __forceinline__ unsigned long long block_token_flags(const uint16_t* 
         return fl;
     }
     if (!hist_clean) {
+        __syncthreads();  // a hinted search of the previous token may still be read by slower warps
         block_clear_key_hist<NT>(hist);
         __syncthreads();
     }
     uint32_t thr;
     int need_eq, tot_eq;
-    if (!(single && hint != kNoKeyHint && block_kth_key_near<DT, NT>(xs, K, k, hint, hist, s, thr, need_eq, tot_eq)))
+    if (!(hint != kNoKeyHint && block_kth_key_near<DT, NT>(xs, K, k, hint, hist, s, thr, need_eq, tot_eq)))
         block_kth_key<NT>(xs, K, k, hist, s, thr, need_eq, tot_eq);
+    if (thr_out != nullptr) *thr_out = thr;
     AFX_MARK(8);
     // Channels above the k-th key are in; of those equal to it, the need_eq lowest ids.  One
     // pass over the thread's chunks, two keys per operation (swar_*), leaves two flag sets in

@@ -118,6 +118,10 @@ class DecoderModel:
     def stats(self) -> torch.Tensor:
         return self._view(afx.BUF_STATS, 0, torch.int32, (self.n_layers, 4, 4))
 
+    @property
+    def hints(self) -> torch.Tensor:
+        return self._view(afx.BUF_HINTS, 0, torch.int32, (self.n_layers, 4, afx.MAX_T))
+
     def layer_step(self, layer: int, pos: int, stream=None):
         afx.afx_layer_step(self.handle, layer, self.state, pos, stream)
 

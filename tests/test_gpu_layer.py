@@ -269,3 +269,45 @@ def test_topk_search_hint_never_changes_the_selection(dt, ties):
         out = run([raw] * 4)
         assert out["stats"][:, 3].tolist() == [0x10000 | e for e in exact], raw
     m.close()
+
+
+@pytest.mark.parametrize("dt", ["bf16", "f16"])
+@pytest.mark.parametrize("T", [2, 4, 8])
+def test_per_token_search_hints_never_change_the_selection(dt, T):
+    """Several tokens per step: each token's top-k search starts from the k-th key its slot
+    recorded last time.  First step without hints, then with its own keys as hints, then with
+    hints that are off by a few keys, at the window's edge, far away, and garbage: every stage
+    still matches the oracle, and the recorded keys are the exact k-th keys of each token."""
+    heads, kvh, max_seq, pos = 4, 2, 48, 37
+    hidden, mlp = heads * 128, 1384
+    cfg = ol.Config(dt, hidden, heads, kvh, mlp, mode=oracle.TOPK)
+    L = synth.layer_weights(35, 0, hidden, heads, kvh, mlp, dt, gain_jitter=0.1)
+    k = [synth.keep_count(K, 50) for K in (hidden, heads * 128, hidden, mlp)]
+    L["k"] = k
+    kc0, vc0 = synth.kv_cache(35, 0, T, max_seq, kvh, pos)
+    L["k_cache"], L["v_cache"] = kc0, vc0
+    h0 = synth.hidden_state(35, 5, T, hidden)
+    lw = oracle_weights(L, k)
+    m = make(cfg, [L], T, afx.MODE_TOPK, max_seq=max_seq)
+    half = 32 if dt == "bf16" else 256
+
+    def run(hints):
+        m.h.copy_(torch.from_numpy(h0).cuda())
+        if hints is not None:
+            m.hints[0, :, :T] = torch.tensor(hints, dtype=torch.int32, device="cuda")
+        m.layer_step(0, pos)
+        torch.cuda.synchronize()
+        return check_layer_stages(cfg, L, lw, m, 0, h0, kc0, vc0, pos, T)
+
+    out = run(None)
+    exact = [[kth_key(out["inputs"][op][t], k[op]) for t in range(T)] for op in range(4)]
+    want = [[0x10000 | e for e in row] for row in exact]
+    assert m.hints.cpu().numpy()[0, :, :T].tolist() == want
+    clamp = lambda v: min(0x7FFF, max(0, v))
+    for delta in (0, 3, -half, half, 7 * half):
+        run([[0x10000 | clamp(e + delta * (1 if t % 2 else -1)) for t, e in enumerate(row)] for row in exact])
+        assert m.hints.cpu().numpy()[0, :, :T].tolist() == want, delta
+    for raw in (0, 0x10000, 0x10000 | 0x7FFF, -1):
+        run([[raw] * T] * 4)
+        assert m.hints.cpu().numpy()[0, :, :T].tolist() == want, raw
+    m.close()
