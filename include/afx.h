@@ -209,7 +209,9 @@ typedef struct {
 } afx_model_desc;
 
 typedef struct {
-    /* DEVICE pointers, channel-contiguous (see the conventions at the top), 16-byte aligned:  */
+    /* DEVICE pointers, channel-contiguous (see the conventions at the top), 16-byte aligned.  */
+    /* A weight pointer may be NULL when that operator is always given another way (host       */
+    /* handles, 4-bit rows); a step that needs it then returns AFX_ERR_INVALID_ARG.            */
     const void* w_qkv;  /* [hidden][(n_heads + 2 n_kv_heads) * 128]  columns: q | k | v        */
     const void* w_o;    /* [n_heads * 128][hidden]                                             */
     const void* w_gu;   /* [hidden][2 * mlp]: columns in groups of 16 = gate[8m..8m+8) then    */
@@ -591,6 +593,29 @@ typedef struct {
 } afx_hosted_ops;
 afx_status afx_layer_step_hosted(afx_model* model, int layer, afx_state* state, int pos, const afx_hosted_ops* ops,
                                  int32_t* dev_status, void* stream);
+
+/*
+ * afx_layer_step for a layer whose operator weights are 4-bit (the storage type of the paper's
+ * models, Sec. 7.1; rows as for afx_sparse_gemv_q4): per operator the input stage + selection
+ * (the side outputs of the fused kernel: normed input, active list, cross-layer bookkeeping),
+ * then the 4-bit sparse GEMV over that list with the operator's epilogue (q|k|v: store; o and
+ * down: h +=; gate|up: silu(gate) * up, rounded to the model's 16-bit type).  One token
+ * (state T == 1).  An operator whose wq is NULL runs fused on the 16-bit weights of the layer
+ * descriptor.  AFX_XL_REUSE models are not supported.
+ *
+ *   wq[op]         DEVICE, 16-byte aligned: K_op rows of ldq_bytes[op] bytes (a multiple of 16,
+ *                  >= afx_q4_row_bytes(N_op)); N_op % 32 == 0.  Borrowed for the call.
+ *   gate|up        block b of 32 outputs of a row holds gate outputs 16b .. 16b+15 in the low
+ *                  4 bits of its 16 bytes and up outputs 16b .. 16b+15 in the high 4 bits: one
+ *                  scale serves 16 gate and 16 up weights of the same intermediate channels.
+ *   dev_status     as for afx_sparse_gemv (may be NULL).
+ */
+typedef struct {
+    const void* wq[4];    /* per AFX_OP_*: 4-bit rows or NULL */
+    int64_t ldq_bytes[4]; /* row stride where wq is given     */
+} afx_q4_layer;
+afx_status afx_layer_step_q4(afx_model* model, int layer, afx_state* state, int pos, const afx_q4_layer* q4,
+                             int32_t* dev_status, void* stream);
 
 /*
  * The MLP block without any allocation (the paper has no counterpart: this entry point exists

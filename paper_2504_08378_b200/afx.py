@@ -113,6 +113,11 @@ class HostedOps(ctypes.Structure):
     _fields_ = [("cache", c_void_p * 4), ("swap", c_void_p * 4), ("slot", c_void_p * 4)]
 
 
+class Q4Layer(ctypes.Structure):
+    """afx_q4_layer"""
+    _fields_ = [("wq", c_void_p * 4), ("ldq_bytes", c_int64 * 4)]
+
+
 class AfxError(RuntimeError):
     def __init__(self, fn: str, status: int):
         self.status = status
@@ -180,6 +185,7 @@ def lib() -> ctypes.CDLL:
         L.afx_sparse_gemv_q4.argtypes = [c_void_p, c_int, c_int, c_int64, c_void_p, c_int, c_void_p, c_void_p, c_void_p,
                                          c_int, c_void_p, c_void_p]
         L.afx_layer_step_hosted.argtypes = [c_void_p, c_int, c_void_p, c_int, ctypes.POINTER(HostedOps), c_void_p, c_void_p]
+        L.afx_layer_step_q4.argtypes = [c_void_p, c_int, c_void_p, c_int, ctypes.POINTER(Q4Layer), c_void_p, c_void_p]
         L.afx_mlp_block_noalloc.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_void_p, c_int, c_int, c_int,
                                             c_float, c_int, c_float, c_void_p, c_void_p]
         _lib = L
@@ -429,6 +435,11 @@ def afx_sparse_gemv_q4(Wq, K: int, N: int, ldq_bytes: int, x, x_dtype, idx, coun
     _check("afx_sparse_gemv_q4",
            lib().afx_sparse_gemv_q4(_ptr(Wq), int(K), int(N), int(ldq_bytes), _ptr(x), _dt(x_dtype), _ptr(idx), _ptr(count),
                                     _ptr(y), int(accumulate), _ptr(dev_status), _stream(stream)))
+
+
+def afx_layer_step_q4(model: int, layer: int, state: int, pos: int, q4: Q4Layer, stream=None, dev_status=None):
+    _check("afx_layer_step_q4", lib().afx_layer_step_q4(model, int(layer), state, int(pos), ctypes.byref(q4),
+                                                        _ptr(dev_status), _stream(stream)))
 
 
 def afx_layer_step_hosted(model: int, layer: int, state: int, pos: int, ops: HostedOps, stream=None, dev_status=None):

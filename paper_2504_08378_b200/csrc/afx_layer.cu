@@ -6,6 +6,7 @@
 #include "afx_attn.cuh"
 #include "afx_fused.cuh"
 #include "afx_launch.cuh"
+#include "afx_q4.cuh"
 
 namespace afx {
 
@@ -172,8 +173,8 @@ extern "C" afx_status afx_model_create(const afx_model_desc* desc, const afx_lay
     const int K_op[4] = {d.hidden, d.n_heads * d.head_dim, d.hidden, d.mlp};
     for (int l = 0; l < d.n_layers; ++l) {
         const afx_layer_desc& L = layers[l];
-        if (L.w_qkv == nullptr || L.w_o == nullptr || L.w_gu == nullptr || L.w_down == nullptr ||
-            L.g_attn == nullptr || L.g_mlp == nullptr || L.k_cache == nullptr || L.v_cache == nullptr)
+        // (a NULL weight pointer is allowed: the operator must then come from a host handle or 4-bit rows)
+        if (L.g_attn == nullptr || L.g_mlp == nullptr || L.k_cache == nullptr || L.v_cache == nullptr)
             return AFX_ERR_INVALID_ARG;
         if (!aligned16(L.w_qkv) || !aligned16(L.w_o) || !aligned16(L.w_gu) || !aligned16(L.w_down) ||
             !aligned16(L.k_cache) || !aligned16(L.v_cache) || !aligned16(L.g_attn) || !aligned16(L.g_mlp))
@@ -354,6 +355,7 @@ static afx_status launch_layer_kernel(afx_model* m, int layer, afx_state* s, int
     a.eps = d.rms_eps;
     switch (which) {
         case AFX_STEP_QKV:  // q | k | v
+            if (L.w_qkv == nullptr) return AFX_ERR_INVALID_ARG;
             a.Wt = static_cast<const uint16_t*>(L.w_qkv);
             a.ldw = m->n_qkv;
             a.K = d.hidden;
@@ -381,6 +383,7 @@ static afx_status launch_layer_kernel(afx_model* m, int layer, afx_state* s, int
             return launch_attention(d.dtype, at, st);
         }
         case AFX_STEP_O:
+            if (L.w_o == nullptr) return AFX_ERR_INVALID_ARG;
             a.Wt = static_cast<const uint16_t*>(L.w_o);
             a.ldw = d.hidden;
             a.K = n_attn;
@@ -390,6 +393,7 @@ static afx_status launch_layer_kernel(afx_model* m, int layer, afx_state* s, int
             plan_selection(m, s, layer, AFX_OP_O, true, &a);
             return launch_fused<IN_X, EP_ACCUM>(d.dtype, a, st);
         case AFX_STEP_GU:  // gate | up, silu(gate) * up
+            if (L.w_gu == nullptr) return AFX_ERR_INVALID_ARG;
             a.Wt = static_cast<const uint16_t*>(L.w_gu);
             a.ldw = 2 * static_cast<int64_t>(d.mlp);
             a.K = d.hidden;
@@ -401,6 +405,7 @@ static afx_status launch_layer_kernel(afx_model* m, int layer, afx_state* s, int
             plan_selection(m, s, layer, AFX_OP_GU, true, &a);
             return launch_fused<IN_NORM, EP_SILU>(d.dtype, a, st);
         case AFX_STEP_DOWN:
+            if (L.w_down == nullptr) return AFX_ERR_INVALID_ARG;
             a.Wt = static_cast<const uint16_t*>(L.w_down);
             a.ldw = d.hidden;
             a.K = d.mlp;
@@ -544,6 +549,76 @@ extern "C" afx_status afx_layer_step_hosted(afx_model* m, int layer, afx_state* 
     return AFX_OK;
 }
 
+extern "C" afx_status afx_layer_step_q4(afx_model* m, int layer, afx_state* s, int pos, const afx_q4_layer* q4,
+                                        int32_t* dev_status, void* stream) {
+    using namespace afx;
+    afx_status rc = check_step(m, layer, s);
+    if (rc != AFX_OK) return rc;
+    if (q4 == nullptr || pos < 0 || pos >= m->d.max_seq) return AFX_ERR_INVALID_ARG;
+    if (m->d.xl_mode == AFX_XL_REUSE || s->T != 1) return AFX_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(dev_status) & 3u) != 0) return AFX_ERR_ALIGNMENT;
+    const afx_model_desc& d = m->d;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int N_op[4] = {m->n_qkv, d.hidden, 2 * d.mlp, d.hidden};
+    for (int op = 0; op < 4; ++op) {
+        if (q4->wq[op] == nullptr) continue;
+        if ((N_op[op] & 31) != 0) return AFX_ERR_UNSUPPORTED;
+        if (!aligned16(q4->wq[op]) || (q4->ldq_bytes[op] & 15) != 0) return AFX_ERR_ALIGNMENT;
+        if (q4->ldq_bytes[op] < static_cast<int64_t>(afx_q4_row_bytes(N_op[op]))) return AFX_ERR_INVALID_ARG;
+    }
+    float* h = reinterpret_cast<float*>(s->blob + s->off_h);
+    float* qkv = reinterpret_cast<float*>(s->blob + s->off_qkv);
+    uint16_t* attn = reinterpret_cast<uint16_t*>(s->blob + s->off_attn);
+    uint16_t* hm = reinterpret_cast<uint16_t*>(s->blob + s->off_hm);
+    int32_t* stats = reinterpret_cast<int32_t*>(s->blob + s->off_stats);
+    const afx_layer_desc& L = m->layers[layer];
+    const int which_of[4] = {AFX_STEP_QKV, AFX_STEP_O, AFX_STEP_GU, AFX_STEP_DOWN};
+    for (int op = 0; op < 4; ++op) {
+        if (op == AFX_OP_O && (rc = launch_layer_kernel(m, layer, s, pos, AFX_STEP_ATTN, st)) != AFX_OK) return rc;
+        if (q4->wq[op] == nullptr) {  // 16-bit weights: the fused kernel
+            if ((rc = launch_layer_kernel(m, layer, s, pos, which_of[op], st)) != AFX_OK) return rc;
+            continue;
+        }
+        // 1. input stage + selection
+        FusedArgs a = {};
+        a.T = 1;
+        a.eps = d.rms_eps;
+        a.K = m->K_op[op];
+        a.ldw = N_op[op];
+        const uint16_t* x16 = nullptr;  // the operator's 16-bit input
+        const bool norm = op == AFX_OP_QKV || op == AFX_OP_GU;
+        if (norm) {
+            a.h = h;
+            a.gain = op == AFX_OP_QKV ? L.g_attn : L.g_mlp;
+            a.xnorm_out = reinterpret_cast<uint16_t*>(s->blob + s->off_xnorm[op == AFX_OP_QKV ? 0 : 1]);
+            x16 = a.xnorm_out;
+        } else {
+            a.x = op == AFX_OP_O ? attn : hm;
+            x16 = a.x;
+        }
+        plan_selection(m, s, layer, op, true, &a);
+        rc = norm ? launch_select_only<IN_NORM>(d.dtype, a, st) : launch_select_only<IN_X>(d.dtype, a, st);
+        if (rc != AFX_OK) return rc;
+        // 2. the operator on the 4-bit rows of the active channels
+        Q4Args g = {};
+        g.Wq = static_cast<const unsigned char*>(q4->wq[op]);
+        g.ldq = q4->ldq_bytes[op];
+        g.K = m->K_op[op];
+        g.N = N_op[op];
+        g.x = x16;
+        g.idx = a.idx_out;
+        g.count = stats + (static_cast<size_t>(layer) * 4 + op) * 4;
+        g.status = dev_status;
+        switch (op) {
+            case AFX_OP_QKV: g.ep = Q4_STORE; g.y = qkv; break;
+            case AFX_OP_GU: g.ep = Q4_SILU; g.out_bits = hm; break;
+            default: g.ep = Q4_ACCUM; g.y = h; break;
+        }
+        if ((rc = launch_q4_list(d.dtype, g, st)) != AFX_OK) return rc;
+    }
+    return AFX_OK;
+}
+
 extern "C" afx_status afx_mlp_block(afx_model* m, int layer, afx_state* s, const void* x, float* y,
                                     void* stream) {
     using namespace afx;
@@ -555,6 +630,7 @@ extern "C" afx_status afx_mlp_block(afx_model* m, int layer, afx_state* s, const
     const afx_layer_desc& L = m->layers[layer];
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     uint16_t* hm = reinterpret_cast<uint16_t*>(s->blob + s->off_hm);
+    if (L.w_gu == nullptr || L.w_down == nullptr) return AFX_ERR_INVALID_ARG;
     FusedArgs a = {};
     a.T = s->T;
     a.eps = d.rms_eps;

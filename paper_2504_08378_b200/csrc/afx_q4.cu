@@ -16,6 +16,7 @@
 #include <cooperative_groups.h>
 
 #include "afx_launch.cuh"
+#include "afx_q4.cuh"
 
 namespace afx {
 
@@ -26,18 +27,6 @@ constexpr int kQ4Warps = kQ4Threads / 32;
 constexpr int kQ4Unroll = 8;   // 8-byte loads in flight per lane
 constexpr int kQ4Cap = 1024;   // staged list entries per pass
 constexpr int kQ4Opl = 16;     // outputs per lane and channel: half a block of 32
-
-struct Q4Args {
-    const unsigned char* Wq;
-    int64_t ldq;  // row stride in bytes (multiple of 16)
-    int K, N;
-    const uint16_t* x;
-    const int32_t* idx;
-    const int32_t* count;
-    float* y;
-    int accumulate;
-    int32_t* status;
-};
 
 __device__ __forceinline__ uint2 ld_stream_8B(const void* p) {
     uint2 v;
@@ -195,12 +184,30 @@ __global__ void __launch_bounds__(kQ4Threads, 2) sparse_gemv_q4_kernel(Q4Args a)
         part[o] = s;
     }
     cluster.sync();
-    for (int o = rank + S * tid; o < PW; o += S * kQ4Threads) {
-        const int out = tile * PW + o;
-        if (out < a.N) {
-            float s = 0.0f;
-            for (int q = 0; q < S; ++q) s += cluster.map_shared_rank(part, q)[o];
-            a.y[out] = a.accumulate ? a.y[out] + s : s;
+    if (a.ep == Q4_SILU) {
+        // pair r of the tile: gate = output 32 * (r / 16) + r % 16, up = 16 further on
+        constexpr int HP = PW / 2;
+        for (int r = rank + S * tid; r < HP; r += S * kQ4Threads) {
+            const int og = (r >> 4) * 32 + (r & 15);
+            const int m = tile * HP + r;
+            if (2 * m < a.N) {
+                float g = 0.0f, u = 0.0f;
+                for (int q = 0; q < S; ++q) {
+                    const float* pq = cluster.map_shared_rank(part, q);
+                    g += pq[og];
+                    u += pq[og + 16];
+                }
+                a.out_bits[m] = float_to_bits<XDT>(g / (1.0f + expf(-g)) * u);
+            }
+        }
+    } else {
+        for (int o = rank + S * tid; o < PW; o += S * kQ4Threads) {
+            const int out = tile * PW + o;
+            if (out < a.N) {
+                float s = 0.0f;
+                for (int q = 0; q < S; ++q) s += cluster.map_shared_rank(part, q)[o];
+                a.y[out] = a.ep == Q4_ACCUM ? a.y[out] + s : s;
+            }
         }
     }
     cluster.sync();  // peers may still be reading this block's sums
@@ -244,6 +251,10 @@ static afx_status launch_q4(const Q4Args& a, cudaStream_t st) {
     }
 }
 
+afx_status launch_q4_list(int x_dtype, const Q4Args& a, cudaStream_t st) {
+    return x_dtype == AFX_F16 ? launch_q4<AFX_F16>(a, st) : launch_q4<AFX_BF16>(a, st);
+}
+
 }  // namespace afx
 
 extern "C" size_t afx_q4_row_bytes(int N) {
@@ -263,7 +274,7 @@ extern "C" afx_status afx_sparse_gemv_q4(const void* Wq, int K, int N, int64_t l
         (reinterpret_cast<uintptr_t>(count) & 3u) != 0 || (reinterpret_cast<uintptr_t>(dev_status) & 3u) != 0)
         return AFX_ERR_ALIGNMENT;
     if (ldq_bytes < static_cast<int64_t>(afx_q4_row_bytes(N))) return AFX_ERR_INVALID_ARG;
-    Q4Args a;
+    Q4Args a = {};
     a.Wq = static_cast<const unsigned char*>(Wq);
     a.ldq = ldq_bytes;
     a.K = K;
@@ -272,8 +283,8 @@ extern "C" afx_status afx_sparse_gemv_q4(const void* Wq, int K, int N, int64_t l
     a.idx = idx;
     a.count = count;
     a.y = y;
-    a.accumulate = accumulate ? 1 : 0;
+    a.ep = accumulate ? Q4_ACCUM : Q4_STORE;
     a.status = dev_status;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    return x_dtype == AFX_F16 ? launch_q4<AFX_F16>(a, st) : launch_q4<AFX_BF16>(a, st);
+    return launch_q4_list(x_dtype, a, st);
 }

@@ -40,14 +40,24 @@ class DecoderModel:
         self.K_op = [hidden, n_heads * head_dim, hidden, mlp]
         self._keep = []
         descs = []
-        self.k_cache, self.v_cache = [], []
+        self.k_cache, self.v_cache, self.q4 = [], [], []
         for L in layers:
             d = afx.LayerDesc()
-            w_gu = L["w_gu"] if "w_gu" in L else synth.interleave_gate_up(L["w_gate"], L["w_up"])
-            tens = dict(w_qkv=to_device_bits(L["w_qkv"]), w_o=to_device_bits(L["w_o"]),
-                        w_gu=to_device_bits(w_gu),
-                        w_down=to_device_bits(L["w_down"]),
+            # 16-bit weights may be absent when the layer is only stepped over 4-bit rows ("q4")
+            w_gu = L.get("w_gu")
+            if w_gu is None and L.get("w_gate") is not None:
+                w_gu = synth.interleave_gate_up(L["w_gate"], L["w_up"])
+            dev = lambda w: None if w is None else to_device_bits(w)
+            tens = dict(w_qkv=dev(L.get("w_qkv")), w_o=dev(L.get("w_o")), w_gu=dev(w_gu), w_down=dev(L.get("w_down")),
                         g_attn=to_device_bits(L["g_attn"]).float(), g_mlp=to_device_bits(L["g_mlp"]).float())
+            q4 = None
+            if L.get("q4") is not None:  # per operator a uint8 CUDA tensor [K_op][row bytes] or None
+                q4 = afx.Q4Layer()
+                for op, rows in enumerate(L["q4"]):
+                    q4.wq[op] = None if rows is None else rows.data_ptr()
+                    q4.ldq_bytes[op] = 0 if rows is None else rows.shape[1]
+                tens["q4"] = L["q4"]
+            self.q4.append(q4)
             if "k_cache" in L:
                 kc, vc = to_device_bits(L["k_cache"]), to_device_bits(L["v_cache"])
             else:
@@ -57,7 +67,8 @@ class DecoderModel:
             self.v_cache.append(vc)
             tens["k_cache"], tens["v_cache"] = kc, vc
             for name, t in tens.items():
-                setattr(d, name, t.data_ptr())
+                if name != "q4":
+                    setattr(d, name, None if t is None else t.data_ptr())
             for op in range(4):
                 d.k[op] = int(L.get("k", [0, 0, 0, 0])[op])
                 d.tau[op] = float(L.get("tau", [0.0, 0.0, 0.0, 0.0])[op])
@@ -131,6 +142,13 @@ class DecoderModel:
     def decode_step(self, pos: int, stream=None):
         for layer in range(self.n_layers):
             afx.afx_layer_step(self.handle, layer, self.state, pos, stream)
+
+    def layer_step_q4(self, layer: int, pos: int, stream=None, dev_status=None):
+        afx.afx_layer_step_q4(self.handle, layer, self.state, pos, self.q4[layer], stream, dev_status)
+
+    def decode_step_q4(self, pos: int, stream=None, dev_status=None):
+        for layer in range(self.n_layers):
+            afx.afx_layer_step_q4(self.handle, layer, self.state, pos, self.q4[layer], stream, dev_status)
 
     def mlp_block(self, layer: int, x: torch.Tensor, y: torch.Tensor, stream=None):
         afx.afx_mlp_block(self.handle, layer, self.state, x, y, stream)

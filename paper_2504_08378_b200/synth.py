@@ -205,6 +205,26 @@ def split_gate_up(w_gu: np.ndarray):
 
 # ---- 4-bit block-quantised weights (the storage type the paper evaluates) ----
 
+def device_q4_weight(seed: int, stream: int, K: int, N: int, sigma: float = 0.02):
+    """q4_weight's recipe drawn with torch's seeded CUDA generator: a uint8 CUDA tensor
+    [K][q4_row_bytes(N)] (rounded normal codes, scales around 2.5 * sigma / 8 with either sign).
+    Input generation only; not the same stream of numbers as q4_weight."""
+    import torch
+    g = torch.Generator(device="cuda")
+    g.manual_seed((int(seed) * 1000003 + int(stream)) & (2**63 - 1))
+    rows = torch.zeros((K, q4_row_bytes(N)), dtype=torch.uint8, device="cuda")
+    step = max(1, (1 << 25) // N)
+    for r0 in range(0, K, step):  # bounded temporaries
+        r1 = min(K, r0 + step)
+        q = torch.randn((r1 - r0, N // 32, 32), generator=g, device="cuda").mul_(8.0 / 2.5).add_(8.0).round_().clamp_(0, 15)
+        q = q.to(torch.uint8)
+        rows[r0:r1, : N // 2] = (q[:, :, :16] | (q[:, :, 16:] << 4)).reshape(r1 - r0, N // 2)
+        d = sigma * 2.5 / 8.0 * (1.0 + 0.1 * torch.randn((r1 - r0, N // 32), generator=g, device="cuda"))
+        d = d * (torch.rand((r1 - r0, N // 32), generator=g, device="cuda") < 0.5).to(torch.float32).mul_(2.0).sub_(1.0)
+        rows[r0:r1, N // 2: N // 2 + N // 16] = d.to(torch.float16).view(torch.uint8)
+    return rows
+
+
 def q4_row_bytes(N: int) -> int:
     """Bytes of one channel of N outputs (N a multiple of 32) in the 4-bit layout: N/2 bytes of
     4-bit codes, then N/32 fp16 block scales, padded to a multiple of 16 bytes."""
