@@ -1108,8 +1108,7 @@ def variant_q4(st, peak):
 
 def variant_q4_step(st, n_layers=32):
     """The 7B decode token with every operator's weights 4-bit (afx_layer_step_q4: per operator
-    the input stage + selection kernel, then the 4-bit sparse GEMV with the operator's
-    epilogue), same selection as the headline (top 50 %, cross-layer depth 3, bookkeeping), a
+    one kernel -- input stage, selection, 4-bit sparse GEMV, epilogue), same selection as the headline (top 50 %, cross-layer depth 3, bookkeeping), a
     different token every replay.  Bytes = active rows * row bytes (codes + scales)."""
     import numpy as np
     import torch
@@ -1156,12 +1155,13 @@ def variant_q4_step(st, n_layers=32):
     w_bytes = n_layers * sum(kk * rb for kk, rb in zip(k, row_bytes))
     kv_bytes = n_layers * 2 * past * heads * 128 * 2
     out = {"workload": f"llama7b_decode_{n_layers}L_q4_top50", "ms_per_step": round(ms, 4), "tokens_per_s": round(1e3 / ms, 2),
-           "kernels_per_step": 9 * n_layers, "device_status": int(status.item()),
+           "kernels_per_step": 5 * n_layers, "device_status": int(status.item()),
            "active_weight_bytes": int(w_bytes), "active_weight_gbs": round(w_bytes / (ms * 1e-3) / 1e9, 1),
            "weights_plus_kv_gbs": round((w_bytes + kv_bytes) / (ms * 1e-3) / 1e9, 1),
            "weight_bytes_resident": int(n_layers * sum(K * rb for (K, _), rb in zip(shapes, row_bytes))),
-           "note": "4-bit rows are 3.56x smaller than bf16 rows; the 4-bit kernel is bound by instruction issue and "
-                   "each operator is two launches (selection, then GEMV), so the token is no faster than with bf16 weights"}
+           "note": "4-bit rows are 3.56x smaller than bf16 rows, but the 4-bit streaming loop is bound by instruction "
+                   "issue (5-6 instructions per weight) and the fixed phases of every operator are those of the bf16 "
+                   "step: the token takes about as long as with bf16 weights, in 0.28 of the memory"}
     m.close()
     del m, layers, g
     torch.cuda.empty_cache()

@@ -596,19 +596,20 @@ afx_status afx_layer_step_hosted(afx_model* model, int layer, afx_state* state, 
 
 /*
  * afx_layer_step for a layer whose operator weights are 4-bit (the storage type of the paper's
- * models, Sec. 7.1; rows as for afx_sparse_gemv_q4): per operator the input stage + selection
- * (the side outputs of the fused kernel: normed input, active list, cross-layer bookkeeping),
- * then the 4-bit sparse GEMV over that list with the operator's epilogue (q|k|v: store; o and
- * down: h +=; gate|up: silu(gate) * up, rounded to the model's 16-bit type).  One token
- * (state T == 1).  An operator whose wq is NULL runs fused on the 16-bit weights of the layer
- * descriptor.  AFX_XL_REUSE models are not supported.
+ * models, Sec. 7.1; rows as for afx_sparse_gemv_q4): per operator ONE kernel, as in
+ * afx_layer_step -- input stage, selection with its side outputs (normed input, active list,
+ * cross-layer bookkeeping), the 4-bit sparse GEMV over the selected channels and the operator's
+ * epilogue (q|k|v: store; o and down: h +=; gate|up: silu(gate) * up, rounded to the model's
+ * 16-bit type).  One token (state T == 1).  An operator whose wq is NULL runs on the 16-bit
+ * weights of the layer descriptor.  AFX_XL_REUSE models are not supported.
  *
  *   wq[op]         DEVICE, 16-byte aligned: K_op rows of ldq_bytes[op] bytes (a multiple of 16,
  *                  >= afx_q4_row_bytes(N_op)); N_op % 32 == 0.  Borrowed for the call.
  *   gate|up        block b of 32 outputs of a row holds gate outputs 16b .. 16b+15 in the low
  *                  4 bits of its 16 bytes and up outputs 16b .. 16b+15 in the high 4 bits: one
  *                  scale serves 16 gate and 16 up weights of the same intermediate channels.
- *   dev_status     as for afx_sparse_gemv (may be NULL).
+ *   dev_status     reserved (may be NULL; 4-byte aligned): every list this path multiplies by
+ *                  comes from its own selection, so no device check can fire.
  */
 typedef struct {
     const void* wq[4];    /* per AFX_OP_*: 4-bit rows or NULL */

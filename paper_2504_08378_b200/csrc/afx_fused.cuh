@@ -6,6 +6,7 @@
 #pragma once
 
 #include "afx_gemv.cuh"
+#include "afx_q4.cuh"
 #include "afx_select.cuh"
 
 namespace afx {
@@ -65,11 +66,15 @@ __host__ __device__ inline size_t fused_dyn_smem(int in_kind, int K, int T) {
     return fused_input_smem(in_kind, K, T) + fused_flag_smem(K) + kKeyHistBytes;
 }
 
-template <int DT, int TMAX, int PW, int CAP, int IN, int EP>
+// WQ4: the weights are 4-bit rows (afx_sparse_gemv_q4's layout; one token): Wt points at them,
+// ldw is the row stride in units of 2 bytes, the tile is PW = 512, 256 or 128 outputs wide and
+// the streaming loop and the reduction are the 4-bit kernel's.
+template <int DT, int TMAX, int PW, int CAP, int IN, int EP, bool WQ4 = false>
 __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char* dyn, SelectScratch* sel,
                                                GemvRecv<TMAX>* recv) {
-    constexpr int LPC = PW / 8;
+    constexpr int LPC = WQ4 ? PW / kQ4Opl : PW / 8;
     static_assert(sizeof(GemvSmem<TMAX, CAP>) <= kKeyHistBytes, "work area too small");
+    static_assert(!WQ4 || (TMAX == 1 && CAP * 8 + (kQ4Warps + 1) * PW * 4 <= kKeyHistBytes), "4-bit: one token, sums behind the staged list");
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int warp = tid >> 5;
@@ -212,7 +217,7 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
     int cnt = 0;
     int pos0 = 0;                  // list position of this thread's first active channel
     unsigned long long fl = 0ull;  // this thread's active flags (own selection)
-    const int out0 = tile * PW + (lane % LPC) * 8;
+    const int out0 = tile * PW + (lane % LPC) * (WQ4 ? kQ4Opl : 8);
     const bool lane_ok = out0 < a.N;
     // One token, top-k: the list length is k whatever x holds, so this block's part
     // [c_lo, c_hi) of the list is known before the selection and the pass that decides the
@@ -299,6 +304,9 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
     for (int t = 0; t < TMAX; ++t)
 #pragma unroll
         for (int q = 0; q < 8; ++q) acc[t][q] = 0.0f;
+    f32x2 qacc[8];  // 4-bit weights: 16 outputs per lane
+#pragma unroll
+    for (int i = 0; i < 8; ++i) qacc[i] = pack_f32x2(0.0f, 0.0f);
 
     const int n_mine = __popcll(fl);
     for (int c0 = c_lo; c0 < c_hi; c0 += CAP) {
@@ -330,14 +338,24 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
         }
         __syncthreads();
         AFX_MARK(4);
-        if (lane_ok)
+        if (WQ4) {
+            if (lane_ok)
+                q4_stream<LPC>(reinterpret_cast<const unsigned char*>(Wt), a.N, out0 / kQ4Opl, sm->col, sm->xv[0], staged, qacc);
+        } else if (lane_ok) {
             gemv_stream<DT, TMAX, PW, CAP, false>(reinterpret_cast<const uint4*>(Wt + out0), T, sm, staged, acc);
+        }
     }
     AFX_MARK(5);
 
     AFX_MARK(6);
 
-    gemv_finish_tile<DT, TMAX, PW, CAP, EP>(acc, T, tile, sm, recv, a.ep);
+    if (WQ4) {
+        cluster_wait();  // pairs with the cluster_arrive() at kernel start
+        q4_finish<DT, LPC>(qacc, reinterpret_cast<float*>(work) + 2 * CAP, tile, a.N,
+                           EP == EP_SILU ? Q4_SILU : (EP == EP_ACCUM ? Q4_ACCUM : Q4_STORE), a.ep.y, a.ep.out_bits);
+    } else {
+        gemv_finish_tile<DT, TMAX, PW, CAP, EP>(acc, T, tile, sm, recv, a.ep);
+    }
     AFX_MARK(7);
 }
 

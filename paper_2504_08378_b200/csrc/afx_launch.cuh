@@ -94,23 +94,23 @@ struct GemvShapeChoice {
 
 // Widest tile and largest cluster such that all tiles' clusters are resident at once
 // (one wave) and the block count is as large as possible.  kerns[i] is the kernel
-// instantiated for tile width 256 >> i.
+// instantiated for tile width widest >> i.
 #ifdef AFX_EXPERIMENT
 extern int g_force_pw, g_force_s;  // experiment knobs (0 = automatic)
 extern int g_cluster_margin;      // experiment knob (< 0 = automatic)
 #endif
 
 inline GemvShapeChoice choose_gemv_shape(int N, const void* const kerns[3], size_t dyn_smem,
-                                         int extra_clusters = 0) {
+                                         int extra_clusters = 0, int widest = 256) {
 #ifdef AFX_EXPERIMENT
     const int force_pw = g_force_pw, force_s = g_force_s, force_margin = g_cluster_margin;
 #else
     constexpr int force_pw = 0, force_s = 0, force_margin = -1;
 #endif
-    GemvShapeChoice best = {64, 1, (N + 63) / 64};
+    GemvShapeChoice best = {widest >> 2, 1, (N + (widest >> 2) - 1) / (widest >> 2)};
     int best_blocks = -1;
     for (int i = 0; i < 3; ++i) {
-        const int pw = 256 >> i;
+        const int pw = widest >> i;
         if (force_pw && pw != force_pw) continue;
         const int tiles = (N + pw - 1) / pw;
         int s_fit = 0;

@@ -26,6 +26,15 @@ fused_op_kernel(FusedArgs a) {
     fused_op_block<DT, TMAX, PW, CAP, IN, EP>(a, dyn, &sel, &recv);
 }
 
+// The one-token operator over 4-bit rows: tiles of PW = 512, 256 or 128 outputs.
+template <int DT, int PW, int IN, int EP>
+__global__ void __launch_bounds__(kGemvThreads, 2) fused_q4_kernel(FusedArgs a) {
+    constexpr int CAP = FusedShape<1>::kStageCap;
+    extern __shared__ __align__(16) unsigned char dyn[];
+    __shared__ SelectScratch sel;
+    fused_op_block<DT, 1, PW, CAP, IN, EP, true>(a, dyn, &sel, nullptr);
+}
+
 template <int DT, int REP>
 __global__ void __launch_bounds__(kAttnThreads, REP <= 2 ? 2 : 1) attention_kernel(AttnArgs a) {
     __shared__ AttnSmem sm;
@@ -62,6 +71,33 @@ static afx_status launch_fused_t(const FusedArgs& a, cudaStream_t st) {
         case 128: return launch_clustered(fused_op_kernel<DT, TMAX, 128, IN, EP>, c.S, rows, dyn, b, st);
         default: return launch_clustered(fused_op_kernel<DT, TMAX, 64, IN, EP>, c.S, rows, dyn, b, st);
     }
+}
+
+// a.Wt = the 4-bit rows, a.ldw = their stride in units of 2 bytes, a.T == 1, a.N % 32 == 0.
+template <int DT, int IN, int EP>
+static afx_status launch_fused_q4_dt(const FusedArgs& a, cudaStream_t st) {
+    if (static_cast<uint64_t>(a.K) * static_cast<uint64_t>(a.ldw >> 3) > 0x100000000ull) return AFX_ERR_CAPACITY;
+    const size_t dyn = fused_dyn_smem(IN, a.K, 1);
+    const void* kerns[3] = {reinterpret_cast<const void*>(fused_q4_kernel<DT, 512, IN, EP>),
+                            reinterpret_cast<const void*>(fused_q4_kernel<DT, 256, IN, EP>),
+                            reinterpret_cast<const void*>(fused_q4_kernel<DT, 128, IN, EP>)};
+    FusedArgs b = a;
+    b.side_cluster = (a.idx_out != nullptr || a.count_out != nullptr || a.bitmap_out != nullptr ||
+                      a.xnorm_out != nullptr || a.bitmap_pred != nullptr || a.kth_slot != nullptr)
+                         ? 1 : 0;
+    const GemvShapeChoice c = choose_gemv_shape(a.N, kerns, dyn, b.side_cluster, 512);
+    if (c.tiles + b.side_cluster > 65535) return AFX_ERR_CAPACITY;
+    const int rows = c.tiles + b.side_cluster;
+    switch (c.pw) {
+        case 512: return launch_clustered(fused_q4_kernel<DT, 512, IN, EP>, c.S, rows, dyn, b, st);
+        case 256: return launch_clustered(fused_q4_kernel<DT, 256, IN, EP>, c.S, rows, dyn, b, st);
+        default: return launch_clustered(fused_q4_kernel<DT, 128, IN, EP>, c.S, rows, dyn, b, st);
+    }
+}
+
+template <int IN, int EP>
+static afx_status launch_fused_q4(int dtype, const FusedArgs& a, cudaStream_t st) {
+    return dtype == AFX_F16 ? launch_fused_q4_dt<AFX_F16, IN, EP>(a, st) : launch_fused_q4_dt<AFX_BF16, IN, EP>(a, st);
 }
 
 template <int DT, int IN, int EP>
@@ -557,6 +593,7 @@ extern "C" afx_status afx_layer_step_q4(afx_model* m, int layer, afx_state* s, i
     if (q4 == nullptr || pos < 0 || pos >= m->d.max_seq) return AFX_ERR_INVALID_ARG;
     if (m->d.xl_mode == AFX_XL_REUSE || s->T != 1) return AFX_ERR_UNSUPPORTED;
     if ((reinterpret_cast<uintptr_t>(dev_status) & 3u) != 0) return AFX_ERR_ALIGNMENT;
+    (void)dev_status;  // every list this path multiplies by comes from its own selection: nothing to report
     const afx_model_desc& d = m->d;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int N_op[4] = {m->n_qkv, d.hidden, 2 * d.mlp, d.hidden};
@@ -570,7 +607,6 @@ extern "C" afx_status afx_layer_step_q4(afx_model* m, int layer, afx_state* s, i
     float* qkv = reinterpret_cast<float*>(s->blob + s->off_qkv);
     uint16_t* attn = reinterpret_cast<uint16_t*>(s->blob + s->off_attn);
     uint16_t* hm = reinterpret_cast<uint16_t*>(s->blob + s->off_hm);
-    int32_t* stats = reinterpret_cast<int32_t*>(s->blob + s->off_stats);
     const afx_layer_desc& L = m->layers[layer];
     const int which_of[4] = {AFX_STEP_QKV, AFX_STEP_O, AFX_STEP_GU, AFX_STEP_DOWN};
     for (int op = 0; op < 4; ++op) {
@@ -579,42 +615,37 @@ extern "C" afx_status afx_layer_step_q4(afx_model* m, int layer, afx_state* s, i
             if ((rc = launch_layer_kernel(m, layer, s, pos, which_of[op], st)) != AFX_OK) return rc;
             continue;
         }
-        // 1. input stage + selection
+        // input stage + selection + the operator on the 4-bit rows of the active channels, one kernel
         FusedArgs a = {};
         a.T = 1;
         a.eps = d.rms_eps;
+        a.Wt = static_cast<const uint16_t*>(q4->wq[op]);
+        a.ldw = q4->ldq_bytes[op] >> 1;
         a.K = m->K_op[op];
-        a.ldw = N_op[op];
-        const uint16_t* x16 = nullptr;  // the operator's 16-bit input
-        const bool norm = op == AFX_OP_QKV || op == AFX_OP_GU;
-        if (norm) {
-            a.h = h;
-            a.gain = op == AFX_OP_QKV ? L.g_attn : L.g_mlp;
-            a.xnorm_out = reinterpret_cast<uint16_t*>(s->blob + s->off_xnorm[op == AFX_OP_QKV ? 0 : 1]);
-            x16 = a.xnorm_out;
-        } else {
-            a.x = op == AFX_OP_O ? attn : hm;
-            x16 = a.x;
-        }
+        a.N = N_op[op];
         plan_selection(m, s, layer, op, true, &a);
-        rc = norm ? launch_select_only<IN_NORM>(d.dtype, a, st) : launch_select_only<IN_X>(d.dtype, a, st);
-        if (rc != AFX_OK) return rc;
-        // 2. the operator on the 4-bit rows of the active channels
-        Q4Args g = {};
-        g.Wq = static_cast<const unsigned char*>(q4->wq[op]);
-        g.ldq = q4->ldq_bytes[op];
-        g.K = m->K_op[op];
-        g.N = N_op[op];
-        g.x = x16;
-        g.idx = a.idx_out;
-        g.count = stats + (static_cast<size_t>(layer) * 4 + op) * 4;
-        g.status = dev_status;
         switch (op) {
-            case AFX_OP_QKV: g.ep = Q4_STORE; g.y = qkv; break;
-            case AFX_OP_GU: g.ep = Q4_SILU; g.out_bits = hm; break;
-            default: g.ep = Q4_ACCUM; g.y = h; break;
+            case AFX_OP_QKV:
+                a.h = h;
+                a.gain = L.g_attn;
+                a.xnorm_out = reinterpret_cast<uint16_t*>(s->blob + s->off_xnorm[0]);
+                a.ep = {qkv, nullptr, N_op[op]};
+                rc = launch_fused_q4<IN_NORM, EP_STORE>(d.dtype, a, st);
+                break;
+            case AFX_OP_GU:
+                a.h = h;
+                a.gain = L.g_mlp;
+                a.xnorm_out = reinterpret_cast<uint16_t*>(s->blob + s->off_xnorm[1]);
+                a.ep = {nullptr, hm, N_op[op]};
+                rc = launch_fused_q4<IN_NORM, EP_SILU>(d.dtype, a, st);
+                break;
+            default:
+                a.x = op == AFX_OP_O ? attn : hm;
+                a.ep = {h, nullptr, N_op[op]};
+                rc = launch_fused_q4<IN_X, EP_ACCUM>(d.dtype, a, st);
+                break;
         }
-        if ((rc = launch_q4_list(d.dtype, g, st)) != AFX_OK) return rc;
+        if (rc != AFX_OK) return rc;
     }
     return AFX_OK;
 }
