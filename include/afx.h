@@ -601,7 +601,7 @@ afx_status afx_layer_step_hosted(afx_model* model, int layer, afx_state* state, 
  * cross-layer bookkeeping), the 4-bit sparse GEMV over the selected channels and the operator's
  * epilogue (q|k|v: store; o and down: h +=; gate|up: silu(gate) * up, rounded to the model's
  * 16-bit type).  One token (state T == 1).  An operator whose wq is NULL runs on the 16-bit
- * weights of the layer descriptor.  AFX_XL_REUSE models are not supported.
+ * weights of the layer descriptor.  Cross-layer modes as in afx_layer_step.
  *
  *   wq[op]         DEVICE, 16-byte aligned: K_op rows of ldq_bytes[op] bytes (a multiple of 16,
  *                  >= afx_q4_row_bytes(N_op)); N_op % 32 == 0.  Borrowed for the call.

@@ -591,7 +591,7 @@ extern "C" afx_status afx_layer_step_q4(afx_model* m, int layer, afx_state* s, i
     afx_status rc = check_step(m, layer, s);
     if (rc != AFX_OK) return rc;
     if (q4 == nullptr || pos < 0 || pos >= m->d.max_seq) return AFX_ERR_INVALID_ARG;
-    if (m->d.xl_mode == AFX_XL_REUSE || s->T != 1) return AFX_ERR_UNSUPPORTED;
+    if (s->T != 1) return AFX_ERR_UNSUPPORTED;
     if ((reinterpret_cast<uintptr_t>(dev_status) & 3u) != 0) return AFX_ERR_ALIGNMENT;
     (void)dev_status;  // every list this path multiplies by comes from its own selection: nothing to report
     const afx_model_desc& d = m->d;

@@ -40,8 +40,14 @@ def gate_up(y):
     return b[:, :, :16].reshape(y.shape[0], -1), b[:, :, 16:].reshape(y.shape[0], -1)
 
 
-def check_q4_stages(cfg, L16, q4rows, use, lw, m, layer, h0, kc0, vc0, pos):
+def check_q4_stages(cfg, L16, q4rows, use, lw, m, layer, h0, kc0, vc0, pos, lists=None):
+    """`lists` (operator name -> index list): the sets the layer must have computed on when it
+    reuses another layer's (cross-layer REUSE)."""
     dt = cfg.dtype
+
+    def expected(op, x_bits):
+        return lists[op] if lists is not None else ol.select(x_bits, cfg, lw, op)
+
     stats = m.stats.cpu().numpy()[layer]
     n_qkv = (cfg.n_heads + 2 * cfg.n_kv_heads) * cfg.head_dim
 
@@ -54,7 +60,7 @@ def check_q4_stages(cfg, L16, q4rows, use, lw, m, layer, h0, kc0, vc0, pos):
     xa_gpu = bits_np(m.bits(afx.BUF_XNORM, afx.OP_QKV))
     assert ulp_close(xa_gpu, oracle.rmsnorm(h0.astype(np.float64), lw.g_attn, cfg.eps, dt))
     idx = m.idx(afx.OP_QKV).cpu().numpy()[: stats[0][0]]
-    assert np.array_equal(idx, ol.select(xa_gpu, cfg, lw, "qkv"))
+    assert np.array_equal(idx, expected("qkv", xa_gpu))
     qkv_gpu = m.qkv.cpu().numpy()
     assert rel_err(qkv_gpu, gemv(0, n_qkv, xa_gpu, idx, L16["w_qkv"])) <= TOL
     # attention on the GPU's own q, k, v
@@ -64,7 +70,7 @@ def check_q4_stages(cfg, L16, q4rows, use, lw, m, layer, h0, kc0, vc0, pos):
     assert rel_err(oracle.decode(attn_gpu, dt), oracle.decode(attn_ref, dt)) <= 2 * 2.0 ** (-8 if dt == "bf16" else -11) + 1e-3
     # o
     idx_o = m.idx(afx.OP_O).cpu().numpy()[: stats[1][0]]
-    assert np.array_equal(idx_o, ol.select(attn_gpu, cfg, lw, "o"))
+    assert np.array_equal(idx_o, expected("o", attn_gpu))
     h1_ref = h0.astype(np.float64) + gemv(1, cfg.hidden, attn_gpu, idx_o, L16["w_o"])
     # gate|up: the normalised input carries the fp32 error of h + W_o a
     xm_gpu = bits_np(m.bits(afx.BUF_XNORM, afx.OP_GU))
@@ -77,7 +83,7 @@ def check_q4_stages(cfg, L16, q4rows, use, lw, m, layer, h0, kc0, vc0, pos):
     xm_err = (h1_err + 8 * EPS32 * np.abs(h1_ref)) * inv * np.abs(lw.g_mlp)
     assert ulp_close(xm_gpu, oracle.rmsnorm(h1_ref, lw.g_mlp, cfg.eps, dt), frac_exact=0.97, dt=dt, abs_err=xm_err)
     idx_gu = m.idx(afx.OP_GU).cpu().numpy()[: stats[2][0]]
-    assert np.array_equal(idx_gu, ol.select(xm_gpu, cfg, lw, "gu"))
+    assert np.array_equal(idx_gu, expected("gu", xm_gpu))
     hm_gpu = bits_np(m.bits(afx.BUF_HM))
     if use[2]:
         g, u = gate_up(oracle.sparse_gemv_q4(q4rows[2], 2 * cfg.mlp, xm_gpu, dt, idx_gu))
@@ -90,7 +96,7 @@ def check_q4_stages(cfg, L16, q4rows, use, lw, m, layer, h0, kc0, vc0, pos):
     assert ulp_close(hm_gpu, oracle.silu_mul(g, u, dt), frac_exact=0.97, dt=dt, abs_err=silu_mul_err(g, u, ag, au))
     # down
     idx_d = m.idx(afx.OP_DOWN).cpu().numpy()[: stats[3][0]]
-    assert np.array_equal(idx_d, ol.select(hm_gpu, cfg, lw, "down"))
+    assert np.array_equal(idx_d, expected("down", hm_gpu))
     h2_ref = h1_ref + gemv(3, cfg.hidden, hm_gpu, idx_d, L16["w_down"])
     assert rel_err(m.h.cpu().numpy(), h2_ref) <= TOL
     return dict(idx=[idx, idx_o, idx_gu, idx_d], kc=bits_np(m.k_cache[layer]), vc=bits_np(m.v_cache[layer]))
@@ -138,6 +144,40 @@ def test_q4_layer_step_every_stage_matches_oracle(dt, heads, kvh, mlp, use):
         prev = out["idx"]
         h = m.h.cpu().numpy().copy()
     assert int(status.item()) == 0
+    m.close()
+
+
+def test_q4_layer_step_reuses_the_predictor_layers_sets():
+    """Four layers at depth 3, REUSE: layers 1 and 2 compute on layer 0's sets, layer 3 selects again."""
+    dt, heads, kvh, mlp, T, max_seq, pos, NL = "bf16", 4, 2, 1024, 1, 32, 20, 4
+    hidden, n_qkv = heads * 128, (heads + 2 * kvh) * 128
+    cfg = ol.Config(dt, hidden, heads, kvh, mlp, mode=oracle.TOPK, xl_depth=3, xl_mode=2)
+    k = [synth.keep_count(K, 50) for K in (hidden, heads * 128, hidden, mlp)]
+    layers, q4, q4dev, caches = [], [], [], []
+    for l in range(NL):
+        L = synth.layer_weights(64, l, hidden, heads, kvh, mlp, dt, gain_jitter=0.1)
+        L["k"] = k
+        kc0, vc0 = synth.kv_cache(64, l, T, max_seq, kvh, pos)
+        L["k_cache"], L["v_cache"] = kc0, vc0
+        layers.append(L)
+        caches.append((kc0, vc0))
+        rows = q4_layer_weights(64, l, hidden, heads * 128, n_qkv, mlp)
+        q4.append(rows)
+        q4dev.append([torch.from_numpy(r).cuda() for r in rows])
+    m = make(cfg, layers, T, afx.MODE_TOPK, xl_depth=3, xl_mode=afx.XL_REUSE, max_seq=max_seq)
+    h = synth.hidden_state(64, 5, T, hidden, scale=4.0, scales_stream=6)
+    m.h.copy_(torch.from_numpy(h).cuda())
+    use = (True, True, True, True)
+    pred = None
+    for l in range(NL):
+        afx.afx_layer_step_q4(m.handle, l, m.state, pos, q4_struct(q4dev[l], use))
+        torch.cuda.synchronize()
+        own = l % 3 == 0
+        out = check_q4_stages(cfg, layers[l], q4[l], use, oracle_weights(layers[l], k), m, l, h, caches[l][0],
+                              caches[l][1], pos, lists=None if own else dict(zip(OPN, pred)))
+        if own:
+            pred = [i.copy() for i in out["idx"]]
+        h = m.h.cpu().numpy().copy()
     m.close()
 
 
