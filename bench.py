@@ -1049,7 +1049,7 @@ def variant_moe(st, n_layers=4):
     us = e0.elapsed_time(e1) * 1e3 / (reps * n)
     nbytes_active = top * 2 * (k_gu * 2 * M + k_down * H)
     return {"workload": "mixtral8x7b_shaped_moe_block_bf16_top2of8_sparsity50", "layers_in_rotation": n_layers,
-            "us_per_block": round(us, 2), "kernels_per_block": 1 + 2 * top, "active_expert_bytes": nbytes_active,
+            "us_per_block": round(us, 2), "kernels_per_block": 4, "active_expert_bytes": nbytes_active,
             "gbs": round(nbytes_active / (us * 1e-6) / 1e9, 1)}
 
 

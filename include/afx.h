@@ -541,8 +541,10 @@ afx_status afx_cost_search(const afx_cost_search_in* in, afx_cost_choice* out);
  *     p = softmax(logits[e_1..e_top]);  y (+)= sum_r p_r * W_down[e_r](silu(W_gate[e_r] x) * W_up[e_r] x)
  *
  * The experts are chosen ON THE DEVICE (no host round trip): the kernels take their weights
- * from DEVICE tables of device pointers, indexed by what the router kernel wrote.  1 + 2*top
- * kernels on `stream`.
+ * from DEVICE tables of device pointers, indexed by what the router kernel wrote.  Four
+ * kernels on `stream`: the router, the chosen experts' gate|up operators side by side in one
+ * grid, their down operators likewise (each weighted output in the workspace), and the sum of
+ * those outputs in the order of the router's choice.
  * ------------------------------------------------------------------------------------------ */
 
 typedef struct {
@@ -560,8 +562,9 @@ typedef struct {
     const void* w_down_table; /* DEVICE array of n_experts DEVICE pointers: [mlp][hidden]         */
 } afx_moe_desc;
 
-/* Bytes of DEVICE workspace afx_moe_block needs (256-byte aligned): router results and the
- * chosen experts' intermediate vectors.  0 for a bad descriptor. */
+/* Bytes of DEVICE workspace afx_moe_block needs (256-byte aligned): router results, the chosen
+ * experts' intermediate vectors and their weighted outputs before they are added up.  0 for a
+ * bad descriptor. */
 size_t afx_moe_workspace_bytes(const afx_moe_desc* desc);
 
 /*

@@ -50,6 +50,12 @@ struct FusedArgs {
     // repeats input stage and selection only to write the side outputs, off the path of the
     // clusters that stream (its other blocks leave at once) ----
     int side_cluster;
+    // ---- several operators of one family in one grid (groups > 1; no side outputs): the
+    // column tiles are `groups` equal runs, run g being an operator of the same shape with
+    // weights wt_table[wt_sel[g]], input x + g * x_stride, outputs ep.y / ep.out_bits +
+    // g * out_stride (elements) and factor ep.scale[g].  Every cluster selects on its run's input. ----
+    int groups;
+    int64_t x_stride, out_stride;
 };
 
 // Dynamic shared memory: [16-bit inputs: T tokens (IN_NORM) or one token (IN_X), each padded
@@ -66,10 +72,11 @@ __host__ __device__ inline size_t fused_dyn_smem(int in_kind, int K, int T) {
     return fused_input_smem(in_kind, K, T) + fused_flag_smem(K) + kKeyHistBytes;
 }
 
+// GRP: the grid may hold several operators of one family (FusedArgs::groups).
 // WQ4: the weights are 4-bit rows (afx_sparse_gemv_q4's layout; one token): Wt points at them,
 // ldw is the row stride in units of 2 bytes, the tile is PW = 512, 256 or 128 outputs wide and
 // the streaming loop and the reduction are the 4-bit kernel's.
-template <int DT, int TMAX, int PW, int CAP, int IN, int EP, bool WQ4 = false>
+template <int DT, int TMAX, int PW, int CAP, int IN, int EP, bool WQ4 = false, bool GRP = false>
 __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char* dyn, SelectScratch* sel,
                                                GemvRecv<TMAX>* recv) {
     constexpr int LPC = WQ4 ? PW / kQ4Opl : PW / 8;
@@ -78,9 +85,16 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int warp = tid >> 5;
-    const int S = gridDim.x, s = blockIdx.x, tile = blockIdx.y;
+    const int S = gridDim.x, s = blockIdx.x;
     const int T = a.T, K = a.K;
     const bool side = a.side_cluster != 0 && blockIdx.y == gridDim.y - 1;  // the cluster without a tile
+    int tile = blockIdx.y, grp = 0;
+    if (GRP && a.groups > 1) {  // (never together with a side cluster)
+        const int per = gridDim.y / a.groups;
+        grp = tile / per;
+        tile -= grp * per;
+    }
+    auto x_of_run = [&]() { return GRP ? a.x + grp * a.x_stride : a.x; };
     if (side && blockIdx.x != 0) return;  // (a block that has left no longer holds back the next grid)
     // writes the side outputs: block 0 of the side cluster, else block (0,0) next to its GEMV work
     const bool scribe = a.side_cluster != 0 ? side : (blockIdx.x == 0 && blockIdx.y == 0);
@@ -209,7 +223,7 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
     // 16-bit input of token t, channel j, once the stage above / below has run
     auto x_at = [&](int t, int j) -> uint16_t {
         if (IN == IN_NORM) return xs[static_cast<size_t>(t) * Kp + j];
-        return T == 1 ? xs[j] : a.x[static_cast<size_t>(t) * K + j];
+        return T == 1 ? xs[j] : x_of_run()[static_cast<size_t>(t) * K + j];
     };
     AFX_MARK(2);
 
@@ -235,7 +249,7 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
             const uint16_t* xt = xs + (IN == IN_NORM ? static_cast<size_t>(t) * Kp : 0);
             if (IN == IN_X) {
                 if (t > 0) __syncthreads();  // the previous token's keys are still being read
-                block_stage_token(a.x + static_cast<size_t>(t) * K, K, xs);
+                block_stage_token(x_of_run() + static_cast<size_t>(t) * K, K, xs);
             }
             if (early) {
                 fl |= block_token_flags<DT, kGemvThreads>(
@@ -261,7 +275,7 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
         }
         if (T > 1) pos0 = block_prefix(__popcll(fl), sel->wtot[2], cnt);
     } else {
-        if (IN == IN_X && T == 1) block_stage_token(a.x, K, xs);
+        if (IN == IN_X && T == 1) block_stage_token(x_of_run(), K, xs);
         cnt = *a.count_in;
         cnt = max(0, min(cnt, K));
     }
@@ -295,7 +309,7 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
         if (side) return;
     }
     AFX_MARK(3);
-    const uint16_t* Wt = a.wt_table != nullptr ? a.wt_table[*a.wt_sel] : a.Wt;
+    const uint16_t* Wt = a.wt_table != nullptr ? a.wt_table[a.wt_sel[GRP ? grp : 0]] : a.Wt;
     const int c_lo = s * cnt / S;  // S <= 8, cnt <= 2^20: no overflow
     const int c_hi = (s + 1) * cnt / S;
 
@@ -349,12 +363,18 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
 
     AFX_MARK(6);
 
+    EpilogueArgs ep = a.ep;
+    if (GRP && a.groups > 1) {
+        if (ep.y != nullptr) ep.y += grp * a.out_stride;
+        if (ep.out_bits != nullptr) ep.out_bits += grp * a.out_stride;
+        if (ep.scale != nullptr) ep.scale += grp;
+    }
     if (WQ4) {
         cluster_wait();  // pairs with the cluster_arrive() at kernel start
         q4_finish<DT, LPC>(qacc, reinterpret_cast<float*>(work) + 2 * CAP, tile, a.N,
-                           EP == EP_SILU ? Q4_SILU : (EP == EP_ACCUM ? Q4_ACCUM : Q4_STORE), a.ep.y, a.ep.out_bits);
+                           EP == EP_SILU ? Q4_SILU : (EP == EP_ACCUM ? Q4_ACCUM : Q4_STORE), ep.y, ep.out_bits);
     } else {
-        gemv_finish_tile<DT, TMAX, PW, CAP, EP>(acc, T, tile, sm, recv, a.ep);
+        gemv_finish_tile<DT, TMAX, PW, CAP, EP>(acc, T, tile, sm, recv, ep);
     }
     AFX_MARK(7);
 }

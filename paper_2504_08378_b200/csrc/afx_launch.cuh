@@ -101,18 +101,18 @@ extern int g_cluster_margin;      // experiment knob (< 0 = automatic)
 #endif
 
 inline GemvShapeChoice choose_gemv_shape(int N, const void* const kerns[3], size_t dyn_smem,
-                                         int extra_clusters = 0, int widest = 256) {
+                                         int extra_clusters = 0, int widest = 256, int groups = 1) {
 #ifdef AFX_EXPERIMENT
     const int force_pw = g_force_pw, force_s = g_force_s, force_margin = g_cluster_margin;
 #else
     constexpr int force_pw = 0, force_s = 0, force_margin = -1;
 #endif
-    GemvShapeChoice best = {widest >> 2, 1, (N + (widest >> 2) - 1) / (widest >> 2)};
+    GemvShapeChoice best = {widest >> 2, 1, groups * ((N + (widest >> 2) - 1) / (widest >> 2))};
     int best_blocks = -1;
     for (int i = 0; i < 3; ++i) {
         const int pw = widest >> i;
         if (force_pw && pw != force_pw) continue;
-        const int tiles = (N + pw - 1) / pw;
+        const int tiles = groups * ((N + pw - 1) / pw);  // (groups operators of N outputs side by side)
         int s_fit = 0;
         for (int S = kMaxCluster; S >= 1; --S) {
             if (force_s && S != force_s) continue;

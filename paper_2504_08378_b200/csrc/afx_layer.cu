@@ -26,6 +26,16 @@ fused_op_kernel(FusedArgs a) {
     fused_op_block<DT, TMAX, PW, CAP, IN, EP>(a, dyn, &sel, &recv);
 }
 
+// The one-token operator for a family of `groups` operators in one grid (mixture of experts).
+template <int DT, int PW, int IN, int EP>
+__global__ void __launch_bounds__(kGemvThreads, 2) fused_family_kernel(FusedArgs a) {
+    constexpr int CAP = FusedShape<1>::kStageCap;
+    extern __shared__ __align__(16) unsigned char dyn[];
+    __shared__ SelectScratch sel;
+    __shared__ GemvRecv<1> recv;
+    fused_op_block<DT, 1, PW, CAP, IN, EP, false, true>(a, dyn, &sel, &recv);
+}
+
 // The one-token operator over 4-bit rows: tiles of PW = 512, 256 or 128 outputs.
 template <int DT, int PW, int IN, int EP>
 __global__ void __launch_bounds__(kGemvThreads, 2) fused_q4_kernel(FusedArgs a) {
@@ -71,6 +81,32 @@ static afx_status launch_fused_t(const FusedArgs& a, cudaStream_t st) {
         case 128: return launch_clustered(fused_op_kernel<DT, TMAX, 128, IN, EP>, c.S, rows, dyn, b, st);
         default: return launch_clustered(fused_op_kernel<DT, TMAX, 64, IN, EP>, c.S, rows, dyn, b, st);
     }
+}
+
+// `groups` operators of one family (weights from a.wt_table through a.wt_sel[g]) in one grid;
+// one token, no side outputs.
+template <int DT, int IN, int EP>
+static afx_status launch_fused_family_dt(const FusedArgs& a, cudaStream_t st) {
+    if (static_cast<uint64_t>(a.K) * static_cast<uint64_t>(a.ldw >> 3) > 0x100000000ull) return AFX_ERR_CAPACITY;
+    if (a.T != 1 || a.groups < 1 || a.wt_table == nullptr || a.wt_sel == nullptr) return AFX_ERR_INVALID_ARG;
+    const size_t dyn = fused_dyn_smem(IN, a.K, 1);
+    const void* kerns[3] = {reinterpret_cast<const void*>(fused_family_kernel<DT, 256, IN, EP>),
+                            reinterpret_cast<const void*>(fused_family_kernel<DT, 128, IN, EP>),
+                            reinterpret_cast<const void*>(fused_family_kernel<DT, 64, IN, EP>)};
+    FusedArgs b = a;
+    b.side_cluster = 0;
+    const GemvShapeChoice c = choose_gemv_shape(a.N, kerns, dyn, 0, 256, a.groups);
+    if (c.tiles > 65535) return AFX_ERR_CAPACITY;
+    switch (c.pw) {
+        case 256: return launch_clustered(fused_family_kernel<DT, 256, IN, EP>, c.S, c.tiles, dyn, b, st);
+        case 128: return launch_clustered(fused_family_kernel<DT, 128, IN, EP>, c.S, c.tiles, dyn, b, st);
+        default: return launch_clustered(fused_family_kernel<DT, 64, IN, EP>, c.S, c.tiles, dyn, b, st);
+    }
+}
+
+template <int IN, int EP>
+static afx_status launch_fused_family(int dtype, const FusedArgs& a, cudaStream_t st) {
+    return dtype == AFX_F16 ? launch_fused_family_dt<AFX_F16, IN, EP>(a, st) : launch_fused_family_dt<AFX_BF16, IN, EP>(a, st);
 }
 
 // a.Wt = the 4-bit rows, a.ldw = their stride in units of 2 bytes, a.T == 1, a.N % 32 == 0.
@@ -784,11 +820,25 @@ moe_router_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ W
     }
 }
 
+// y[i] (+)= sum over the chosen experts r, in order, of their weighted down projections part[r][i].
+__global__ void __launch_bounds__(256) moe_combine_kernel(const float* __restrict__ part, int64_t stride, int top, int n,
+                                                          int accumulate, float* __restrict__ y) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    float s = accumulate ? y[i] : 0.0f;
+    for (int r = 0; r < top; ++r) s += part[r * stride + i];
+    y[i] = s;
+}
+
+static size_t moe_hm_stride(const afx_moe_desc& d) { return align256(static_cast<size_t>(d.mlp) * 2); }      // bytes
+static size_t moe_part_stride(const afx_moe_desc& d) { return align256(static_cast<size_t>(d.hidden) * 4); }  // bytes
+
 }  // namespace afx
 
 extern "C" size_t afx_moe_workspace_bytes(const afx_moe_desc* d) {
     if (d == nullptr || d->mlp < 8 || d->top < 1 || d->top > afx::kMoeMaxTop) return 0;
-    return afx::align256(sizeof(afx::MoeWork)) + static_cast<size_t>(d->top) * afx::align256(static_cast<size_t>(d->mlp) * 2);
+    if (d->hidden < 8) return 0;
+    return afx::align256(sizeof(afx::MoeWork)) + static_cast<size_t>(d->top) * (afx::moe_hm_stride(*d) + afx::moe_part_stride(*d));
 }
 
 extern "C" afx_status afx_moe_block(const afx_moe_desc* desc, const void* x, float* y, int accumulate, void* workspace,
@@ -821,35 +871,41 @@ extern "C" afx_status afx_moe_block(const afx_moe_desc* desc, const void* x, flo
     else
         moe_router_kernel<AFX_BF16><<<1, kMoeThreads, 0, st>>>(xb, wr, d.ld_router, d.hidden, d.n_experts, d.top, w);
     if (cudaGetLastError() != cudaSuccess) return AFX_ERR_CUDA;
+    // the chosen experts' gate | up operators in one grid (the same input, one silu(gate) * up vector each)
+    float* part = reinterpret_cast<float*>(hm_base + static_cast<size_t>(d.top) * moe_hm_stride(d));
     afx_status rc;
-    for (int r = 0; r < d.top; ++r) {
-        uint16_t* hm = reinterpret_cast<uint16_t*>(hm_base + static_cast<size_t>(r) * align256(static_cast<size_t>(d.mlp) * 2));
-        FusedArgs a = {};
-        a.T = 1;
-        a.mode = d.select_mode;
-        a.wt_sel = &w->sel[r];
-        // gate | up of the r-th chosen expert
-        a.wt_table = reinterpret_cast<const uint16_t* const*>(d.w_gu_table);
-        a.ldw = 2 * static_cast<int64_t>(d.mlp);
-        a.K = d.hidden;
-        a.N = 2 * d.mlp;
-        a.x = xb;
-        a.k = d.k_gu;
-        a.tau = d.tau_gu;
-        a.ep = {nullptr, hm, 2 * d.mlp, nullptr};
-        if ((rc = launch_fused<IN_X, EP_SILU>(d.dtype, a, st)) != AFX_OK) return rc;
-        // its down projection, weighted
-        a.wt_table = reinterpret_cast<const uint16_t* const*>(d.w_down_table);
-        a.ldw = d.hidden;
-        a.K = d.mlp;
-        a.N = d.hidden;
-        a.x = hm;
-        a.k = d.k_down;
-        a.tau = d.tau_down;
-        a.ep = {y, nullptr, d.hidden, &w->weight[r]};
-        rc = (accumulate || r > 0) ? launch_fused<IN_X, EP_ACCUM>(d.dtype, a, st) : launch_fused<IN_X, EP_STORE>(d.dtype, a, st);
-        if (rc != AFX_OK) return rc;
-    }
+    FusedArgs a = {};
+    a.T = 1;
+    a.mode = d.select_mode;
+    a.wt_sel = &w->sel[0];
+    a.groups = d.top;
+    a.wt_table = reinterpret_cast<const uint16_t* const*>(d.w_gu_table);
+    a.ldw = 2 * static_cast<int64_t>(d.mlp);
+    a.K = d.hidden;
+    a.N = 2 * d.mlp;
+    a.x = xb;
+    a.x_stride = 0;
+    a.k = d.k_gu;
+    a.tau = d.tau_gu;
+    a.ep = {nullptr, reinterpret_cast<uint16_t*>(hm_base), 2 * d.mlp, nullptr};
+    a.out_stride = static_cast<int64_t>(moe_hm_stride(d) / 2);
+    if ((rc = launch_fused_family<IN_X, EP_SILU>(d.dtype, a, st)) != AFX_OK) return rc;
+    // their down projections in one grid, each on the active channels of its own input and
+    // weighted by its routing weight, into one partial output per expert
+    a.wt_table = reinterpret_cast<const uint16_t* const*>(d.w_down_table);
+    a.ldw = d.hidden;
+    a.K = d.mlp;
+    a.N = d.hidden;
+    a.x = reinterpret_cast<const uint16_t*>(hm_base);
+    a.x_stride = static_cast<int64_t>(moe_hm_stride(d) / 2);
+    a.k = d.k_down;
+    a.tau = d.tau_down;
+    a.ep = {part, nullptr, d.hidden, &w->weight[0]};
+    a.out_stride = static_cast<int64_t>(moe_part_stride(d) / 4);
+    if ((rc = launch_fused_family<IN_X, EP_STORE>(d.dtype, a, st)) != AFX_OK) return rc;
+    // the experts' contributions meet in the order of the router's choice
+    moe_combine_kernel<<<(d.hidden + 255) / 256, 256, 0, st>>>(part, a.out_stride, d.top, d.hidden, accumulate ? 1 : 0, y);
+    if (cudaGetLastError() != cudaSuccess) return AFX_ERR_CUDA;
     return AFX_OK;
 }
 
