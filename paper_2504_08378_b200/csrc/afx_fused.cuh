@@ -59,17 +59,18 @@ struct FusedArgs {
 };
 
 // Dynamic shared memory: [16-bit inputs: T tokens (IN_NORM) or one token (IN_X), each padded
-// to a multiple of 8 elements] [ceil(K/32) flag words, padded to 16 bytes] [work area: the key
+// to a multiple of 8 elements] [T bitmaps of ceil(K/32) flag words, each padded to 16 bytes: where
+// the blocks of a cluster exchange the per-token sets they decided] [work area: the key
 // histogram during the selection, then the GEMV staging and reduction buffers].
 __host__ __device__ inline size_t fused_input_smem(int in_kind, int K, int T) {
     const size_t Kp = (static_cast<size_t>(K) + 7) / 8 * 8;
     return (in_kind == IN_NORM ? static_cast<size_t>(T) : 1) * Kp * 2;
 }
-__host__ __device__ inline size_t fused_flag_smem(int K) {
-    return (static_cast<size_t>((K + 31) / 32) * 4 + 15) / 16 * 16;
+__host__ __device__ inline size_t fused_flag_smem(int K, int T = 1) {
+    return static_cast<size_t>(T) * ((static_cast<size_t>((K + 31) / 32) * 4 + 15) / 16 * 16);
 }
 __host__ __device__ inline size_t fused_dyn_smem(int in_kind, int K, int T) {
-    return fused_input_smem(in_kind, K, T) + fused_flag_smem(K) + kKeyHistBytes;
+    return fused_input_smem(in_kind, K, T) + fused_flag_smem(K, T) + kKeyHistBytes;
 }
 
 // GRP: the grid may hold several operators of one family (FusedArgs::groups).
@@ -102,7 +103,7 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
 
     const int Kp = (K + 7) & ~7;
     uint16_t* xs = reinterpret_cast<uint16_t*>(dyn);
-    unsigned char* work = dyn + fused_input_smem(IN, K, T) + fused_flag_smem(K);
+    unsigned char* work = dyn + fused_input_smem(IN, K, T) + fused_flag_smem(K, T);
     uint32_t* hist = reinterpret_cast<uint32_t*>(work);
     GemvSmem<TMAX, CAP>* sm = reinterpret_cast<GemvSmem<TMAX, CAP>*>(work);
     float* red16 = reinterpret_cast<float*>(sel->hist);  // block reduction of the norm
@@ -243,17 +244,27 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
     static_assert(TMAX > 1 || kXchgFits, "work area too small for the chunk exchange");
     uint32_t* xchg = kXchgFits ? reinterpret_cast<uint32_t*>(work + kXchgOffset) : nullptr;
     bool first_staged = false;
+    // Several tokens: the blocks of a cluster share the work -- block s decides the sets of the
+    // tokens t with t % S == s and writes their flags into every block's table of per-token
+    // bitmaps (distributed shared memory); after one cluster barrier every thread reads the
+    // union for its own chunks.  (The side cluster works alone and decides every token.)
+    const bool share = TMAX > 1 && T > 1 && own && !side && S > 1;
+    uint8_t* const ftab = dyn + fused_input_smem(IN, K, T);
+    const size_t fstride = fused_flag_smem(K);
     if (own) {
         const int e_lo = s * a.k / S, e_n = min(CAP, (s + 1) * a.k / S - e_lo);
+        if (share) cluster_wait();  // pairs with the cluster_arrive() at kernel start: the peers are running
+        bool first = true;
         for (int t = 0; t < T; ++t) {
+            if (share && t % S != s) continue;
             const uint16_t* xt = xs + (IN == IN_NORM ? static_cast<size_t>(t) * Kp : 0);
             if (IN == IN_X) {
-                if (t > 0) __syncthreads();  // the previous token's keys are still being read
+                if (!first) __syncthreads();  // the previous token's keys are still being read
                 block_stage_token(x_of_run() + static_cast<size_t>(t) * K, K, xs);
             }
             if (early) {
                 fl |= block_token_flags<DT, kGemvThreads>(
-                    xt, K, a.mode, a.k, a.tau, hist, t == 0, sel, true, pos0, cnt, [&](int j, int pos, uint16_t bits) {
+                    xt, K, a.mode, a.k, a.tau, hist, first, sel, true, pos0, cnt, [&](int j, int pos, uint16_t bits) {
                         const int p = pos - e_lo;
                         if (p >= 0 && p < e_n) {  // the histogram is dead by now: its memory is the staging area
                             sm->col[p] = static_cast<uint32_t>(j) * ld16;
@@ -268,10 +279,31 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
 #pragma unroll
                 for (int u = 0; u < TMAX; ++u)
                     if (u == t) h_t = hint_t[u];
-                fl |= block_token_flags<DT, kGemvThreads>(xt, K, a.mode, a.k, a.tau, hist, t == 0, sel, T == 1,
-                                                          pos0, cnt, NoEmit(), 0, 0x7FFFFFFF, h_t, nullptr, &thr_t);
+                const unsigned long long ft =
+                    block_token_flags<DT, kGemvThreads>(xt, K, a.mode, a.k, a.tau, hist, first, sel, T == 1, pos0, cnt,
+                                                        NoEmit(), 0, 0x7FFFFFFF, h_t, nullptr, &thr_t);
                 if (scribe && tid == 0 && topk && T > 1 && a.kth_multi != nullptr) a.kth_multi[t] = 0x10000 | thr_t;
+                if (share) {
+                    int q_lo, q_hi;
+                    thread_chunk_range(K, q_lo, q_hi);
+                    for (int q = 0; q < S; ++q) {
+                        uint8_t* dst = cg::this_cluster().map_shared_rank(ftab + static_cast<size_t>(t) * fstride, q);
+                        for (int c = q_lo; c < q_hi; ++c) dst[c] = static_cast<uint8_t>(ft >> (8 * (c - q_lo)));
+                    }
+                } else {
+                    fl |= ft;
+                }
             }
+            first = false;
+        }
+        if (share) {
+            cluster_arrive();  // the flags written above are visible to the peers after their wait
+            cluster_wait();
+            int q_lo, q_hi;
+            thread_chunk_range(K, q_lo, q_hi);
+            for (int t = 0; t < T; ++t)
+                for (int c = q_lo; c < q_hi; ++c)
+                    fl |= static_cast<unsigned long long>(ftab[static_cast<size_t>(t) * fstride + c]) << (8 * (c - q_lo));
         }
         if (T > 1) pos0 = block_prefix(__popcll(fl), sel->wtot[2], cnt);
     } else {
@@ -374,7 +406,7 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
         q4_finish<DT, LPC>(qacc, reinterpret_cast<float*>(work) + 2 * CAP, tile, a.N,
                            EP == EP_SILU ? Q4_SILU : (EP == EP_ACCUM ? Q4_ACCUM : Q4_STORE), ep.y, ep.out_bits);
     } else {
-        gemv_finish_tile<DT, TMAX, PW, CAP, EP>(acc, T, tile, sm, recv, ep);
+        gemv_finish_tile<DT, TMAX, PW, CAP, EP>(acc, T, tile, sm, recv, ep, !share);
     }
     AFX_MARK(7);
 }
