@@ -6,12 +6,15 @@
 #pragma once
 
 #include "afx_gemv.cuh"
+#include "afx_mma.cuh"
 #include "afx_q4.cuh"
 #include "afx_select.cuh"
 
 namespace afx {
 
 enum { IN_X = 0, IN_NORM = 1 };
+
+constexpr int kFusedMtStages = 6;  // pipeline stages of the several-token operator (one block per SM)
 
 struct FusedArgs {
     const uint16_t* Wt;
@@ -69,19 +72,22 @@ __host__ __device__ inline size_t fused_input_smem(int in_kind, int K, int T) {
 __host__ __device__ inline size_t fused_flag_smem(int K, int T = 1) {
     return static_cast<size_t>(T) * ((static_cast<size_t>((K + 31) / 32) * 4 + 15) / 16 * 16);
 }
-__host__ __device__ inline size_t fused_dyn_smem(int in_kind, int K, int T) {
-    return fused_input_smem(in_kind, K, T) + fused_flag_smem(K, T) + kKeyHistBytes;
+// work = bytes of the work area: the key histogram, or more where the streaming stage needs more
+__host__ __device__ inline size_t fused_dyn_smem(int in_kind, int K, int T, size_t work = kKeyHistBytes) {
+    return fused_input_smem(in_kind, K, T) + fused_flag_smem(K, T) + (work > kKeyHistBytes ? work : kKeyHistBytes);
 }
 
 // GRP: the grid may hold several operators of one family (FusedArgs::groups).
+// WMT: several tokens, the streaming stage runs on the tensor cores (afx_mma.cuh): PW = 256, the
+// work area holds an MtSmem once the selection is over.
 // WQ4: the weights are 4-bit rows (afx_sparse_gemv_q4's layout; one token): Wt points at them,
 // ldw is the row stride in units of 2 bytes, the tile is PW = 512, 256 or 128 outputs wide and
 // the streaming loop and the reduction are the 4-bit kernel's.
-template <int DT, int TMAX, int PW, int CAP, int IN, int EP, bool WQ4 = false, bool GRP = false>
+template <int DT, int TMAX, int PW, int CAP, int IN, int EP, bool WQ4 = false, bool GRP = false, bool WMT = false>
 __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char* dyn, SelectScratch* sel,
                                                GemvRecv<TMAX>* recv) {
     constexpr int LPC = WQ4 ? PW / kQ4Opl : PW / 8;
-    static_assert(sizeof(GemvSmem<TMAX, CAP>) <= kKeyHistBytes, "work area too small");
+    static_assert(WMT || sizeof(GemvSmem<TMAX, CAP>) <= kKeyHistBytes, "work area too small");
     static_assert(!WQ4 || (TMAX == 1 && CAP * 8 + (kQ4Warps + 1) * PW * 4 <= kKeyHistBytes), "4-bit: one token, sums behind the staged list");
     const int tid = threadIdx.x;
     const int lane = tid & 31;
@@ -355,6 +361,46 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
     for (int i = 0; i < 8; ++i) qacc[i] = pack_f32x2(0.0f, 0.0f);
 
     const int n_mine = __popcll(fl);
+    if (WMT) {
+        using MtT = MtSmem<CAP, kFusedMtStages>;
+        MtT* mt = reinterpret_cast<MtT*>(work);
+        constexpr int kMtCap = CAP;
+        float c4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        const uint4* wtile16 = reinterpret_cast<const uint4*>(Wt + static_cast<size_t>(tile) * kMtTile);
+        const int n_chunks = min(kMtTile, a.N - tile * kMtTile) >> 3;
+        for (int c0 = c_lo; c0 < c_hi; c0 += kMtCap) {
+            const int staged = min(kMtCap, c_hi - c0);
+            __syncthreads();  // the work area is free: the histogram / the previous pass has been read
+            if (own) {
+                if (pos0 < c0 + staged && pos0 + n_mine > c0) {
+                    for_each_owned_active(fl, K, pos0, [&](int j, int pos) {
+                        const int p = pos - c0;
+                        if (p >= 0 && p < staged) {
+                            mt->col[p] = static_cast<uint32_t>(j) * ld16;
+#pragma unroll
+                            for (int t = 0; t < TMAX; ++t)
+                                if (t < T) mt->xb[t][p] = x_at(t, j);
+                        }
+                    });
+                }
+            } else {
+                for (int i = tid; i < staged; i += kGemvThreads) {
+                    const int j = a.idx_in[c0 + i];
+                    mt->col[i] = static_cast<uint32_t>(j) * ld16;
+#pragma unroll
+                    for (int t = 0; t < TMAX; ++t)
+                        if (t < T) mt->xb[t][i] = x_at(t, j);
+                }
+            }
+            mt_pad_inputs(mt, T, staged);
+            __syncthreads();
+            mt_stream_pass<DT>(wtile16, mt, staged, n_chunks, c4);
+        }
+        EpilogueArgs ep = a.ep;
+        if (!share) cluster_wait();  // pairs with the cluster_arrive() at kernel start
+        mt_finish<DT>(c4, mt, T, tile, a.N, EP, ep);
+        return;
+    }
     for (int c0 = c_lo; c0 < c_hi; c0 += CAP) {
         const int staged = min(CAP, c_hi - c0);
         if (!(first_staged && c0 == c_lo)) {

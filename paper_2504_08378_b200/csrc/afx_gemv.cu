@@ -1,5 +1,6 @@
 // afx_sparse_gemv: host-side shape selection and launch.
 #include "afx_launch.cuh"
+#include "afx_mma.cuh"
 
 namespace afx {
 
@@ -16,6 +17,32 @@ sparse_gemv_kernel(GemvListArgs a) {
     __shared__ GemvSmem<TMAX, CAP> sm;
     __shared__ GemvRecv<TMAX> recv;
     gemv_list_block<DT, TMAX, PW, CAP>(a, &sm, &recv);
+}
+
+// A few tokens at once: the tensor-core kernel (afx_mma.cuh).  2048 staged entries per pass
+// still leave room for two blocks per SM.
+using MtListSmem = MtSmem<2048, 4>;
+template <int DT>
+__global__ void __launch_bounds__(kGemvThreads, 2) sparse_gemm_mt_kernel(GemvListArgs a) {
+    extern __shared__ __align__(16) unsigned char mt_dyn[];
+    mt_list_block<DT>(a, reinterpret_cast<MtListSmem*>(mt_dyn));
+}
+
+template <int DT>
+static afx_status launch_gemm_mt(const GemvListArgs& a, cudaStream_t st) {
+    const void* kern = reinterpret_cast<const void*>(sparse_gemm_mt_kernel<DT>);
+    const size_t dyn = sizeof(MtListSmem);
+    const int tiles = (a.N + kMtTile - 1) / kMtTile;
+    if (tiles > 65535) return AFX_ERR_CAPACITY;
+    // the largest cluster that keeps every tile's cluster resident at once (a margin stays free, as for the fp32 kernels)
+    const int margin = (tiles + 15) / 16 < 2 ? 2 : (tiles + 15) / 16;
+    int S = 1;
+    for (int s = kMaxCluster; s > 1; --s)
+        if (max_active_clusters(kern, s, dyn) >= tiles + margin) {
+            S = s;
+            break;
+        }
+    return launch_clustered(sparse_gemm_mt_kernel<DT>, S, tiles, dyn, a, st);
 }
 
 int sm_count() {
@@ -51,9 +78,7 @@ static afx_status launch_gemv_t(const GemvListArgs& a, cudaStream_t st) {
 template <int DT>
 static afx_status launch_gemv(const GemvListArgs& a, cudaStream_t st) {
     if (a.T <= 1) return launch_gemv_t<DT, 1>(a, st);
-    if (a.T <= 2) return launch_gemv_t<DT, 2>(a, st);
-    if (a.T <= 4) return launch_gemv_t<DT, 4>(a, st);
-    return launch_gemv_t<DT, 8>(a, st);
+    return launch_gemm_mt<DT>(a, st);
 }
 
 afx_status launch_list_gemv(int dtype, const GemvListArgs& a, cudaStream_t st) {

@@ -26,6 +26,19 @@ fused_op_kernel(FusedArgs a) {
     fused_op_block<DT, TMAX, PW, CAP, IN, EP>(a, dyn, &sel, &recv);
 }
 
+// The operator for several tokens per step: the streaming stage runs on the tensor cores.  The
+// block is alone on its SM: staged entries per pass as many as the inputs of TMAX tokens leave room for.
+template <int TMAX>
+struct FusedMtCap {
+    static constexpr int value = TMAX <= 4 ? 2048 : 1024;
+};
+template <int DT, int TMAX, int IN, int EP>
+__global__ void __launch_bounds__(kGemvThreads, 1) fused_mt_kernel(FusedArgs a) {
+    extern __shared__ __align__(16) unsigned char dyn[];
+    __shared__ SelectScratch sel;
+    fused_op_block<DT, TMAX, kMtTile, FusedMtCap<TMAX>::value, IN, EP, false, false, true>(a, dyn, &sel, nullptr);
+}
+
 // The one-token operator for a family of `groups` operators in one grid (mixture of experts).
 template <int DT, int PW, int IN, int EP>
 __global__ void __launch_bounds__(kGemvThreads, 2) fused_family_kernel(FusedArgs a) {
@@ -136,11 +149,34 @@ static afx_status launch_fused_q4(int dtype, const FusedArgs& a, cudaStream_t st
     return dtype == AFX_F16 ? launch_fused_q4_dt<AFX_F16, IN, EP>(a, st) : launch_fused_q4_dt<AFX_BF16, IN, EP>(a, st);
 }
 
+template <int DT, int TMAX, int IN, int EP>
+static afx_status launch_fused_mt(const FusedArgs& a, cudaStream_t st) {
+    if (static_cast<uint64_t>(a.K) * static_cast<uint64_t>(a.ldw >> 3) > 0x100000000ull) return AFX_ERR_CAPACITY;
+    const void* kern = reinterpret_cast<const void*>(fused_mt_kernel<DT, TMAX, IN, EP>);
+    const size_t dyn = fused_dyn_smem(IN, a.K, a.T, sizeof(MtSmem<FusedMtCap<TMAX>::value, kFusedMtStages>));
+    FusedArgs b = a;
+    b.side_cluster = (a.idx_out != nullptr || a.count_out != nullptr || a.bitmap_out != nullptr ||
+                      a.xnorm_out != nullptr || a.bitmap_pred != nullptr || a.kth_slot != nullptr ||
+                      a.kth_multi != nullptr)
+                         ? 1 : 0;
+    const int tiles = (a.N + kMtTile - 1) / kMtTile;
+    const int rows = tiles + b.side_cluster;
+    if (rows > 65535) return AFX_ERR_CAPACITY;
+    const int margin = (tiles + 15) / 16 < 2 ? 2 : (tiles + 15) / 16;
+    int S = 1;
+    for (int s = kMaxCluster; s > 1; --s)
+        if (max_active_clusters(kern, s, dyn) >= rows + margin) {
+            S = s;
+            break;
+        }
+    return launch_clustered(fused_mt_kernel<DT, TMAX, IN, EP>, S, rows, dyn, b, st);
+}
+
 template <int DT, int IN, int EP>
 static afx_status launch_fused_dt(const FusedArgs& a, cudaStream_t st) {
     if (a.T <= 1) return launch_fused_t<DT, 1, IN, EP>(a, st);
-    if (a.T <= 4) return launch_fused_t<DT, 4, IN, EP>(a, st);
-    return launch_fused_t<DT, 8, IN, EP>(a, st);
+    if (a.T <= 4) return launch_fused_mt<DT, 4, IN, EP>(a, st);
+    return launch_fused_mt<DT, 8, IN, EP>(a, st);
 }
 
 template <int IN, int EP>
@@ -308,8 +344,10 @@ extern "C" afx_status afx_state_create(const afx_model* model, int T, void* blob
         return AFX_ERR_CAPACITY;
     }
     // the widest input stage must fit one block's shared memory
-    const size_t dyn_max = afx::fused_dyn_smem(afx::IN_NORM, model->d.hidden, T);
-    if (dyn_max > 200 * 1024 || model->d.mlp > afx::kSelectFastMaxK ||
+    const size_t dyn_max = afx::fused_dyn_smem(afx::IN_NORM, model->d.hidden, T,
+                                               T > 4 ? sizeof(afx::MtSmem<1024, afx::kFusedMtStages>)
+                                                     : (T > 1 ? sizeof(afx::MtSmem<2048, afx::kFusedMtStages>) : 0));
+    if (dyn_max > 220 * 1024 || model->d.mlp > afx::kSelectFastMaxK ||
         model->d.n_heads * model->d.head_dim > afx::kSelectFastMaxK) {
         delete s;
         return AFX_ERR_UNSUPPORTED;
