@@ -474,6 +474,7 @@ def run_afx(args):
         variants["config1_single_projection"] = variant_config1(st)
         variants["config2_mlp_block_7b_threshold_sweep"] = variant_config2(st)
         variants["config4_llama13b_step"] = variant_config4(st)
+        variants["few_token_sparse_gemv"] = variant_few_tokens(st, peak)
         variants["q4_sparse_gemv"] = variant_q4(st, peak)
         variants["q4_decode_step_7b"] = variant_q4_step(st)
         variants["mixtral_shaped_moe_block"] = variant_moe(st)
@@ -1106,6 +1107,57 @@ def variant_q4(st, peak):
     return out
 
 
+def variant_few_tokens(st, peak, Ts=(1, 2, 4, 8), n_mat=8):
+    """afx_sparse_gemv (list given) and afx_select_gemv (selection + GEMV in one kernel) with
+    several tokens per call at the 13B gate|up shape (5120 -> 27648, bf16, top 40 % per token,
+    union over the tokens), 8 distinct matrices in rotation.  T = 1 runs on the fp32 pipe, T >= 2
+    on the tensor cores.  Bytes = union count * N * 2."""
+    import numpy as np
+    import torch
+    from paper_2504_08378_b200 import afx, synth
+    K, N, dt = 5120, 27648, "bf16"
+    k = synth.keep_count(K, 60)
+    Ws = [synth.device_normal_bits(4, 50 + i, (K, N), 0.02, dt) for i in range(n_mat)]
+
+    def timeit(fn, reps=5):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(st):
+            fn(0)
+            st.synchronize()
+            with torch.cuda.graph(g, stream=st):
+                for i in range(n_mat):
+                    fn(i)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            for _ in range(3):
+                g.replay()
+            e0.record(st)
+            for _ in range(reps):
+                g.replay()
+            e1.record(st)
+        e1.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / (reps * n_mat)
+
+    out = {"workload": "llama13b_gate_up_5120x27648_bf16_top40_union", "points": []}
+    for T in Ts:
+        x = torch.from_numpy(synth.laplace_bits(8, 200, (T, K), dt).view(np.int16)).cuda()
+        idx = torch.empty(K, dtype=torch.int32, device="cuda")
+        cnt = torch.zeros(1, dtype=torch.int32, device="cuda")
+        afx.afx_select_active(x, dt, K, T, afx.MODE_TOPK, k, 0.0, idx, cnt, None)
+        torch.cuda.synchronize()
+        c = int(cnt.item())
+        y = torch.empty((T, N), dtype=torch.float32, device="cuda")
+        us_list = timeit(lambda i: afx.afx_sparse_gemv(Ws[i], dt, K, N, N, x, T, idx, cnt, None, y, 0, stream=st))
+        us_sel = timeit(lambda i: afx.afx_select_gemv(Ws[i], dt, K, N, N, x, T, afx.MODE_TOPK, k, 0.0, y, 0, stream=st))
+        nbytes = c * N * 2
+        out["points"].append({"T": T, "union_count": c, "bytes": nbytes, "pipe": "fp32" if T == 1 else "tensor",
+                              "list_given_us": round(us_list, 2), "list_given_gbs": round(nbytes / us_list / 1e3, 1),
+                              "list_given_frac_of_measured_hbm": round(nbytes / us_list / 1e3 / peak, 4),
+                              "select_gemv_us": round(us_sel, 2), "select_gemv_gbs": round(nbytes / us_sel / 1e3, 1)})
+    del Ws
+    torch.cuda.empty_cache()
+    return out
+
+
 def variant_q4_step(st, n_layers=32):
     """The 7B decode token with every operator's weights 4-bit (afx_layer_step_q4: per operator
     one kernel -- input stage, selection, 4-bit sparse GEMV, epilogue), same selection as the headline (top 50 %, cross-layer depth 3, bookkeeping), a
@@ -1205,7 +1257,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-variants", action="store_true", help="skip the threshold / reuse variants")
     ap.add_argument("--layers", type=int, default=0, help="run only the first N layers (profiling aid)")
-    ap.add_argument("--workload", default="decode7b", choices=["decode7b", "cache70b", "swap70b", "q4", "q4step"],
+    ap.add_argument("--workload", default="decode7b", choices=["decode7b", "cache70b", "swap70b", "q4", "q4step", "fewtok"],
                     help="decode7b: the headline decode token; cache70b: host-resident weights behind the LFU cache; "
                          "swap70b: host-resident weights with cross-layer-group preloading")
     ap.add_argument("--swap-tokens", type=int, default=5, help="tokens of the swap70b workload (the first one warms up)")
@@ -1221,6 +1273,12 @@ def main():
         import torch
         torch.cuda.set_device(0)
         print(json.dumps(variant_q4(torch.cuda.Stream(), measured_peaks()[0]["hbm_gbs"])))
+    elif args.workload == "fewtok":  # several tokens per call at the 13B gate|up shape (--layers N: N matrices, T = 4 only)
+        import torch
+        torch.cuda.set_device(0)
+        small = args.layers > 0
+        print(json.dumps(variant_few_tokens(torch.cuda.Stream(), measured_peaks()[0]["hbm_gbs"],
+                                            Ts=(4,) if small else (1, 2, 4, 8), n_mat=args.layers or 8)))
     elif args.workload == "q4step":  # the decode token over 4-bit weights
         import torch
         torch.cuda.set_device(0)
