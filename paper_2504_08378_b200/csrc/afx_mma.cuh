@@ -44,10 +44,9 @@ static_assert(kMtTokens * kMtPartStride * 4 <= kMtStageBytes, "partial sums reus
 __device__ __forceinline__ uint32_t mt_smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
-// 16 bytes global -> shared; src_bytes = 0 writes zeros and reads nothing
-__device__ __forceinline__ void mt_copy16(void* dst, const void* src, uint32_t src_bytes) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(mt_smem_u32(dst)), "l"(src), "r"(src_bytes)
-                 : "memory");
+// 16 bytes global -> shared (dst = shared-window address); src_bytes = 0 writes zeros and reads nothing
+__device__ __forceinline__ void mt_copy16(uint32_t dst, const void* src, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
 }
 __device__ __forceinline__ void mt_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
@@ -67,64 +66,70 @@ __device__ __forceinline__ void mt_mma(float (&c)[4], const uint32_t (&a)[4], ui
                      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-// Requests the rows of the staged channels [p0, p0 + kMtStageRows) of this tile into `buf`
-// (entries at or beyond `staged` and 16-byte pieces beyond the operator's last output: zeros).
-// wtile16 = the weights at this tile's first output; n_chunks = valid 16-byte pieces per row.
-template <class SMT>
-__device__ __forceinline__ void mt_request_stage(const uint4* wtile16, const SMT* sm, unsigned char* buf, int p0,
-                                                 int staged, int n_chunks) {
-    constexpr int kChunks = kMtTile / 8;
-#pragma unroll
-    for (int i = 0; i < kMtStageRows * kChunks / kGemvThreads; ++i) {
-        const int e = threadIdx.x + i * kGemvThreads;
-        const int row = e / kChunks, ch = e % kChunks;
-        const int p = p0 + row;
-        const bool valid = p < staged && ch < n_chunks;
-        const uint4* src = valid ? wtile16 + sm->col[p] + ch : wtile16;
-        mt_copy16(buf + row * kMtRowBytes + ch * 16, src, valid ? 16u : 0u);
-    }
-}
-
-// c += W^T[16 outputs of this warp][kMtStageRows channels of buf] . X[those channels][8 tokens]
-template <int DT, class SMT>
-__device__ __forceinline__ void mt_multiply_stage(const unsigned char* buf, const SMT* sm, int p0, float (&c)[4]) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int gid = lane >> 2, tig = lane & 3;
-    // lane l gives the address of row l % 8 of matrix l / 8: matrices (channels 0-7 | 8-15) x (outputs 0-7 | 8-15)
-    const uint32_t a_addr = mt_smem_u32(buf) + ((lane >> 4) * 8 + (lane & 7)) * kMtRowBytes +
-                            (warp * 16 + ((lane >> 3) & 1) * 8) * 2;
-    const uint16_t* xrow = &sm->xb[gid][p0 + 2 * tig];
-#pragma unroll
-    for (int k0 = 0; k0 < kMtStageRows; k0 += 16) {
-        uint32_t a[4];
-        asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                     : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3])
-                     : "r"(a_addr + k0 * kMtRowBytes));
-        const uint32_t b0 = *reinterpret_cast<const uint32_t*>(xrow + k0);
-        const uint32_t b1 = *reinterpret_cast<const uint32_t*>(xrow + k0 + 8);
-        mt_mma<DT>(c, a, b0, b1);
-    }
-}
-
 // One pass over the staged channels [0, staged) (sm->col, sm->xb filled, zero x behind `staged`
-// up to the end of the last stage, a block barrier since): kStages - 1 stages of kMtStageRows channels
-// in flight.  Every thread of the block calls it; on return all copies have landed.
+// up to the end of the last stage, a block barrier since): kStages - 1 stages of kMtStageRows
+// channels in flight while one is multiplied.  wtile16 = the weights at this tile's first output;
+// n_chunks = valid 16-byte pieces per row of the tile (pieces beyond the operator's last output
+// and rows at or beyond `staged` are filled with zeros).  Every thread of the block calls it; on
+// return all copies have landed.  Everything that does not depend on the stage is computed once:
+// a thread copies the same 16-byte piece of two rows of every stage, a lane reads the same
+// fragment positions of every stage.
 template <int DT, class SMT>
 __device__ __forceinline__ void mt_stream_pass(const uint4* wtile16, SMT* sm, int staged, int n_chunks, float (&c)[4]) {
-    constexpr int kMtStages = SMT::kStages;
+    constexpr int kSt = SMT::kStages;
+    constexpr int kChunks = kMtTile / 8;                       // 16-byte pieces per row
+    constexpr int kSweep = kGemvThreads / kChunks;             // rows the block copies at once
+    static_assert(kChunks == 32 && kMtStageRows % kSweep == 0, "copy pattern");
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int gid = lane >> 2, tig = lane & 3;
+    const int r0 = tid / kChunks, ch = tid % kChunks;
+    const bool ch_ok = ch < n_chunks;
+    const uint4* src_base = wtile16 + ch;
+    const uint32_t w_base = mt_smem_u32(sm->w[0]);
+    const uint32_t dst0 = w_base + r0 * kMtRowBytes + ch * 16;
+    // lane l gives the address of row l % 8 of matrix l / 8: matrices (channels 0-7 | 8-15) x (outputs 0-7 | 8-15)
+    const uint32_t a0 = w_base + ((lane >> 4) * 8 + (lane & 7)) * kMtRowBytes + (warp * 16 + ((lane >> 3) & 1) * 8) * 2;
+    const uint32_t x0 = mt_smem_u32(&sm->xb[gid][2 * tig]);
     const int n_st = (staged + kMtStageRows - 1) / kMtStageRows;
+
+    auto request = [&](int q, int buf) {
+        if (q < n_st) {
 #pragma unroll
-    for (int q = 0; q < kMtStages - 1; ++q) {
-        if (q < n_st) mt_request_stage(wtile16, sm, sm->w[q], q * kMtStageRows, staged, n_chunks);
+            for (int i = 0; i < kMtStageRows / kSweep; ++i) {
+                const int p = q * kMtStageRows + r0 + i * kSweep;
+                const bool valid = ch_ok && p < staged;
+                const uint4* src = valid ? src_base + sm->col[p] : wtile16;
+                mt_copy16(dst0 + buf * kMtStageBytes + i * kSweep * kMtRowBytes, src, valid ? 16u : 0u);
+            }
+        }
         mt_commit();
-    }
-    for (int q = 0; q < n_st; ++q) {
-        mt_wait<kMtStages - 2>();  // stage q has landed (this thread's copies)
-        __syncthreads();           // ... everybody's; and stage q - 1 has been multiplied by everybody
-        const int nq = q + kMtStages - 1;
-        if (nq < n_st) mt_request_stage(wtile16, sm, sm->w[nq % kMtStages], nq * kMtStageRows, staged, n_chunks);
-        mt_commit();
-        mt_multiply_stage<DT>(sm->w[q % kMtStages], sm, q * kMtStageRows, c);
+    };
+    auto multiply = [&](int q, int buf) {
+#pragma unroll
+        for (int k0 = 0; k0 < kMtStageRows; k0 += 16) {
+            uint32_t a[4], b0, b1;
+            asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                         : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3])
+                         : "r"(a0 + buf * kMtStageBytes + k0 * kMtRowBytes));
+            const uint32_t xa = x0 + (q * kMtStageRows + k0) * 2;
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(b0) : "r"(xa));
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(b1) : "r"(xa + 16));
+            mt_mma<DT>(c, a, b0, b1);
+        }
+    };
+#pragma unroll
+    for (int j = 0; j < kSt - 1; ++j) request(j, j);
+    for (int q0 = 0; q0 < n_st; q0 += kSt) {
+#pragma unroll
+        for (int j = 0; j < kSt; ++j) {  // stage q0 + j lives in buffer j
+            const int q = q0 + j;
+            if (q < n_st) {
+                mt_wait<kSt - 2>();  // stage q has landed (this thread's copies)
+                __syncthreads();     // ... everybody's; and stage q - 1 has been multiplied by everybody
+                request(q + kSt - 1, (j + kSt - 1) % kSt);
+                multiply(q, j);
+            }
+        }
     }
     mt_wait<0>();
 }
