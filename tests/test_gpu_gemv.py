@@ -183,3 +183,73 @@ def test_select_gemv_hint_slot(dt):
         assert int(slot.item()) == 0x10000 | exact, preset
         assert int(cnt_d.item()) == k and np.array_equal(idx_d.cpu().numpy()[:k], want), preset
         assert rel_err(y.cpu().numpy(), y_ref) <= TOL, preset
+
+
+@pytest.mark.parametrize("dt", ["f16", "bf16"])
+@pytest.mark.parametrize("T,K,N,n_active", [
+    (2, 40, 8, 0), (2, 40, 8, 1), (3, 300, 264, 31), (5, 300, 264, 33),      # one narrow tile + a ragged one; lists around one 32-channel stage
+    (4, 5000, 520, 2049), (8, 5000, 520, 4100),                              # more entries than one staged pass holds (2 and 3 passes)
+    (7, 777, 1376, 777), (2, 2048, 2304 + 8, 1000),                          # every channel active; several tiles and a tail
+])
+def test_several_tokens_on_the_tensor_cores_edges(dt, T, K, N, n_active):
+    """afx_sparse_gemv with 2..8 tokens multiplies on the tensor cores: lists that end inside a
+    16-channel step, empty lists, passes beyond the staged capacity, ragged last tiles, token
+    counts that leave rows of the 8-token operand empty."""
+    Wt = synth.weight(210, T, K, N, dt)
+    x = synth.laplace_bits(211, T, (T, K), dt)
+    idx = np.sort(np.random.default_rng(K + n_active).choice(K, n_active, replace=False)).astype(np.int32)
+    y = run_gemv(Wt, dt, N, x, idx)
+    ref = oracle.sparse_gemv(Wt, dt, N, x, idx)
+    if n_active == 0:
+        assert not y.any()
+    else:
+        assert rel_err(y, ref) <= TOL
+    y0 = synth.laplace(212, T, (T, N)).astype(np.float32)
+    assert rel_err(run_gemv(Wt, dt, N, x, idx, y0=y0), ref + y0) <= TOL
+    assert np.array_equal(run_gemv(Wt, dt, N, x, idx), y), "the same inputs give the same bits"
+
+
+def test_several_tokens_slot_list_bad_entries_and_nan_inputs():
+    """The several-token kernel keeps the list kernel's rules: slot indirection, skipped entries
+    reported through the status word, and a NaN input of a channel that is NOT in the list, or a
+    NaN weight row nobody asked for, never reaches y (rows behind the list's end are zero-filled
+    in shared memory and meet zero inputs)."""
+    dt, T, K, N = "bf16", 4, 200, 264
+    Wt = synth.weight(213, 1, K, N, dt)
+    x = synth.laplace_bits(213, 2, (T, K), dt)
+    good = np.array([3, 10, 11, 50, 95, 96, 130, 199], np.int32)
+    x[:, 7] = 0x7FC0  # NaN inputs at channels outside the list
+    x[:, 150] = 0xFF80  # -inf
+    guard = 4
+    buf = torch.full((K + 2 * guard, N), -1, dtype=torch.int16, device="cuda")  # 0xFFFF = a NaN pattern
+    buf[guard:guard + K] = dev_bits(Wt)
+    W = buf[guard:guard + K]
+    y = torch.empty((T, N), dtype=torch.float32, device="cuda")
+
+    def gemv(idx, count, slot=None, rows=W):
+        st = torch.zeros(1, dtype=torch.int32, device="cuda")
+        afx.afx_sparse_gemv(rows, dt, K, N, N, dev_bits(x), T, dev_i32(idx), dev_i32([count]),
+                            None if slot is None else dev_i32(slot), y, 0, dev_status=st)
+        torch.cuda.synchronize()
+        return int(st.item()), y.cpu().numpy()
+
+    ref = oracle.sparse_gemv(Wt, dt, N, x, good)
+    st, out = gemv(good, good.size)
+    assert st == 0 and np.isfinite(out).all() and rel_err(out, ref) <= TOL
+    st, out = gemv(np.array([3, -1, 10, 11, 50, 200, 95, 96, 1 << 30, 130, 199], np.int32), 11)
+    assert st == 1 and np.isfinite(out).all() and rel_err(out, ref) <= TOL
+    # slots: the listed channels' rows sit permuted in a small cache; two of them found no row
+    perm = np.array([5, 2, 7, 0, 1, 6, 3, 4], np.int32)
+    cache = np.full((8, N), 0xFFFF, np.uint16)
+    cache[perm] = Wt[good]
+    slot = perm.copy()
+    slot[[1, 6]] = -1
+    keep = np.array([0, 2, 3, 4, 5, 7])
+    st, out = gemv(good, good.size, slot, rows=dev_bits(cache))
+    assert st == 3 and np.isfinite(out).all()
+    assert rel_err(out, oracle.sparse_gemv(Wt, dt, N, x, good[keep])) <= TOL
+    full = np.arange(K, dtype=np.int32)
+    full = full[(full != 7) & (full != 150)]
+    padded = np.concatenate([full, np.full(K - full.size, 3, np.int32)])  # K entries: the count is clamped to K
+    st, out = gemv(padded, K + 9)
+    assert st == 3 and np.isfinite(out).all()
