@@ -14,8 +14,6 @@ namespace afx {
 
 enum { IN_X = 0, IN_NORM = 1 };
 
-constexpr int kFusedMtStages = 6;  // pipeline stages of the several-token operator (one block per SM)
-
 struct FusedArgs {
     const uint16_t* Wt;
     // mixture of experts: if wt_table is given, the weights are wt_table[*wt_sel] (both DEVICE;
@@ -78,16 +76,16 @@ __host__ __device__ inline size_t fused_dyn_smem(int in_kind, int K, int T, size
 }
 
 // GRP: the grid may hold several operators of one family (FusedArgs::groups).
-// WMT: several tokens, the streaming stage runs on the tensor cores (afx_mma.cuh): PW = 256, the
-// work area holds an MtSmem once the selection is over.
+// WMT > 0: several tokens, the streaming stage runs on the tensor cores (afx_mma.cuh) with WMT
+// pipeline stages: PW = 256, the work area holds an MtSmem<CAP, WMT> once the selection is over.
 // WQ4: the weights are 4-bit rows (afx_sparse_gemv_q4's layout; one token): Wt points at them,
 // ldw is the row stride in units of 2 bytes, the tile is PW = 512, 256 or 128 outputs wide and
 // the streaming loop and the reduction are the 4-bit kernel's.
-template <int DT, int TMAX, int PW, int CAP, int IN, int EP, bool WQ4 = false, bool GRP = false, bool WMT = false>
+template <int DT, int TMAX, int PW, int CAP, int IN, int EP, bool WQ4 = false, bool GRP = false, int WMT = 0>
 __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char* dyn, SelectScratch* sel,
                                                GemvRecv<TMAX>* recv) {
     constexpr int LPC = WQ4 ? PW / kQ4Opl : PW / 8;
-    static_assert(WMT || sizeof(GemvSmem<TMAX, CAP>) <= kKeyHistBytes, "work area too small");
+    static_assert(WMT > 0 || sizeof(GemvSmem<TMAX, CAP>) <= kKeyHistBytes, "work area too small");
     static_assert(!WQ4 || (TMAX == 1 && CAP * 8 + (kQ4Warps + 1) * PW * 4 <= kKeyHistBytes), "4-bit: one token, sums behind the staged list");
     const int tid = threadIdx.x;
     const int lane = tid & 31;
@@ -362,7 +360,7 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
 
     const int n_mine = __popcll(fl);
     if (WMT) {
-        using MtT = MtSmem<CAP, kFusedMtStages>;
+        using MtT = MtSmem<CAP, (WMT > 0 ? WMT : 2)>;
         MtT* mt = reinterpret_cast<MtT*>(work);
         constexpr int kMtCap = CAP;
         float c4[4] = {0.0f, 0.0f, 0.0f, 0.0f};

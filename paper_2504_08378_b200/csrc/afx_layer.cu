@@ -32,11 +32,11 @@ template <int TMAX>
 struct FusedMtCap {
     static constexpr int value = TMAX <= 4 ? 2048 : 1024;
 };
-template <int DT, int TMAX, int IN, int EP>
+template <int DT, int TMAX, int IN, int EP, int STAGES>
 __global__ void __launch_bounds__(kGemvThreads, 1) fused_mt_kernel(FusedArgs a) {
     extern __shared__ __align__(16) unsigned char dyn[];
     __shared__ SelectScratch sel;
-    fused_op_block<DT, TMAX, kMtTile, FusedMtCap<TMAX>::value, IN, EP, false, false, true>(a, dyn, &sel, nullptr);
+    fused_op_block<DT, TMAX, kMtTile, FusedMtCap<TMAX>::value, IN, EP, false, false, STAGES>(a, dyn, &sel, nullptr);
 }
 
 // The one-token operator for a family of `groups` operators in one grid (mixture of experts).
@@ -149,11 +149,15 @@ static afx_status launch_fused_q4(int dtype, const FusedArgs& a, cudaStream_t st
     return dtype == AFX_F16 ? launch_fused_q4_dt<AFX_F16, IN, EP>(a, st) : launch_fused_q4_dt<AFX_BF16, IN, EP>(a, st);
 }
 
-template <int DT, int TMAX, int IN, int EP>
-static afx_status launch_fused_mt(const FusedArgs& a, cudaStream_t st) {
-    if (static_cast<uint64_t>(a.K) * static_cast<uint64_t>(a.ldw >> 3) > 0x100000000ull) return AFX_ERR_CAPACITY;
-    const void* kern = reinterpret_cast<const void*>(fused_mt_kernel<DT, TMAX, IN, EP>);
-    const size_t dyn = fused_dyn_smem(IN, a.K, a.T, sizeof(MtSmem<FusedMtCap<TMAX>::value, kFusedMtStages>));
+// Pipeline stages of the several-token operator: 6 (one block per SM has the room), 3 where the
+// tokens' inputs leave less (wide models with 8 tokens).
+constexpr int kFusedMtStages = 6, kFusedMtStagesSmall = 3;
+constexpr size_t kMaxDynSmem = 227 * 1024;
+
+template <int DT, int TMAX, int IN, int EP, int STAGES>
+static afx_status launch_fused_mt_st(const FusedArgs& a, cudaStream_t st) {
+    const void* kern = reinterpret_cast<const void*>(fused_mt_kernel<DT, TMAX, IN, EP, STAGES>);
+    const size_t dyn = fused_dyn_smem(IN, a.K, a.T, sizeof(MtSmem<FusedMtCap<TMAX>::value, STAGES>));
     FusedArgs b = a;
     b.side_cluster = (a.idx_out != nullptr || a.count_out != nullptr || a.bitmap_out != nullptr ||
                       a.xnorm_out != nullptr || a.bitmap_pred != nullptr || a.kth_slot != nullptr ||
@@ -169,7 +173,17 @@ static afx_status launch_fused_mt(const FusedArgs& a, cudaStream_t st) {
             S = s;
             break;
         }
-    return launch_clustered(fused_mt_kernel<DT, TMAX, IN, EP>, S, rows, dyn, b, st);
+    return launch_clustered(fused_mt_kernel<DT, TMAX, IN, EP, STAGES>, S, rows, dyn, b, st);
+}
+
+template <int DT, int TMAX, int IN, int EP>
+static afx_status launch_fused_mt(const FusedArgs& a, cudaStream_t st) {
+    if (static_cast<uint64_t>(a.K) * static_cast<uint64_t>(a.ldw >> 3) > 0x100000000ull) return AFX_ERR_CAPACITY;
+    if (fused_dyn_smem(IN, a.K, a.T, sizeof(MtSmem<FusedMtCap<TMAX>::value, kFusedMtStages>)) <= kMaxDynSmem)
+        return launch_fused_mt_st<DT, TMAX, IN, EP, kFusedMtStages>(a, st);
+    if (fused_dyn_smem(IN, a.K, a.T, sizeof(MtSmem<FusedMtCap<TMAX>::value, kFusedMtStagesSmall>)) <= kMaxDynSmem)
+        return launch_fused_mt_st<DT, TMAX, IN, EP, kFusedMtStagesSmall>(a, st);
+    return AFX_ERR_CAPACITY;
 }
 
 template <int DT, int IN, int EP>
@@ -344,10 +358,11 @@ extern "C" afx_status afx_state_create(const afx_model* model, int T, void* blob
         return AFX_ERR_CAPACITY;
     }
     // the widest input stage must fit one block's shared memory
-    const size_t dyn_max = afx::fused_dyn_smem(afx::IN_NORM, model->d.hidden, T,
-                                               T > 4 ? sizeof(afx::MtSmem<1024, afx::kFusedMtStages>)
-                                                     : (T > 1 ? sizeof(afx::MtSmem<2048, afx::kFusedMtStages>) : 0));
-    if (dyn_max > 220 * 1024 || model->d.mlp > afx::kSelectFastMaxK ||
+    const size_t dyn_max = afx::fused_dyn_smem(
+        afx::IN_NORM, model->d.hidden, T,
+        T > 4 ? sizeof(afx::MtSmem<afx::FusedMtCap<8>::value, afx::kFusedMtStagesSmall>)
+              : (T > 1 ? sizeof(afx::MtSmem<afx::FusedMtCap<4>::value, afx::kFusedMtStagesSmall>) : 0));
+    if (dyn_max > afx::kMaxDynSmem || model->d.mlp > afx::kSelectFastMaxK ||
         model->d.n_heads * model->d.head_dim > afx::kSelectFastMaxK) {
         delete s;
         return AFX_ERR_UNSUPPORTED;

@@ -121,6 +121,16 @@ def test_config4_13b_layer(T):
     _run_layers(cfg, [dev], [host], k, T, 2048, 2056, 4)
 
 
+def test_wide_model_with_eight_tokens_per_step():
+    """Hidden size 8192 with 8 tokens: the normalised inputs of 8 tokens take 128 KB of shared
+    memory, so the several-token operators run with their short pipeline."""
+    dt, hidden, heads, kvh, mlp = "bf16", 8192, 64, 8, 2048
+    cfg = ol.Config(dt, hidden, heads, kvh, mlp, mode=oracle.TOPK)
+    k = [synth.keep_count(K, 50) for K in (hidden, heads * 128, hidden, mlp)]
+    dev, host = full_layer(7, 0, hidden, heads, kvh, mlp, dt, k=k)
+    _run_layers(cfg, [dev], [host], k, 8, 40, 48, 7)
+
+
 def test_config5_70b_layer_and_cached_down_projection():
     dt, hidden, heads, kvh, mlp = "bf16", 8192, 64, 8, 28672
     cfg = ol.Config(dt, hidden, heads, kvh, mlp, mode=oracle.TOPK)
