@@ -28,15 +28,18 @@ fused_op_kernel(FusedArgs a) {
 
 // The operator for several tokens per step: the streaming stage runs on the tensor cores.  The
 // block is alone on its SM: staged entries per pass as many as the inputs of TMAX tokens leave room for.
+constexpr int kFusedMtStages = 6, kFusedMtStagesSmall = 3;  // pipeline stages of the several-token operator
+constexpr size_t kMaxDynSmem = 227 * 1024;
 template <int TMAX>
 struct FusedMtCap {
     static constexpr int value = TMAX <= 4 ? 2048 : 1024;
 };
-template <int DT, int TMAX, int IN, int EP, int STAGES>
-__global__ void __launch_bounds__(kGemvThreads, 1) fused_mt_kernel(FusedArgs a) {
+// CAPM staged entries per pass, STAGES pipeline stages, BPS blocks per SM.
+template <int DT, int TMAX, int IN, int EP, int STAGES, int CAPM, int BPS>
+__global__ void __launch_bounds__(kGemvThreads, BPS) fused_mt_kernel(FusedArgs a) {
     extern __shared__ __align__(16) unsigned char dyn[];
     __shared__ SelectScratch sel;
-    fused_op_block<DT, TMAX, kMtTile, FusedMtCap<TMAX>::value, IN, EP, false, false, STAGES>(a, dyn, &sel, nullptr);
+    fused_op_block<DT, TMAX, kMtTile, CAPM, IN, EP, false, false, STAGES>(a, dyn, &sel, nullptr);
 }
 
 // The one-token operator for a family of `groups` operators in one grid (mixture of experts).
@@ -149,15 +152,11 @@ static afx_status launch_fused_q4(int dtype, const FusedArgs& a, cudaStream_t st
     return dtype == AFX_F16 ? launch_fused_q4_dt<AFX_F16, IN, EP>(a, st) : launch_fused_q4_dt<AFX_BF16, IN, EP>(a, st);
 }
 
-// Pipeline stages of the several-token operator: 6 (one block per SM has the room), 3 where the
-// tokens' inputs leave less (wide models with 8 tokens).
-constexpr int kFusedMtStages = 6, kFusedMtStagesSmall = 3;
-constexpr size_t kMaxDynSmem = 227 * 1024;
 
-template <int DT, int TMAX, int IN, int EP, int STAGES>
+template <int DT, int TMAX, int IN, int EP, int STAGES, int CAPM, int BPS>
 static afx_status launch_fused_mt_st(const FusedArgs& a, cudaStream_t st) {
-    const void* kern = reinterpret_cast<const void*>(fused_mt_kernel<DT, TMAX, IN, EP, STAGES>);
-    const size_t dyn = fused_dyn_smem(IN, a.K, a.T, sizeof(MtSmem<FusedMtCap<TMAX>::value, STAGES>));
+    const void* kern = reinterpret_cast<const void*>(fused_mt_kernel<DT, TMAX, IN, EP, STAGES, CAPM, BPS>);
+    const size_t dyn = fused_dyn_smem(IN, a.K, a.T, sizeof(MtSmem<CAPM, STAGES>));
     FusedArgs b = a;
     b.side_cluster = (a.idx_out != nullptr || a.count_out != nullptr || a.bitmap_out != nullptr ||
                       a.xnorm_out != nullptr || a.bitmap_pred != nullptr || a.kth_slot != nullptr ||
@@ -173,16 +172,22 @@ static afx_status launch_fused_mt_st(const FusedArgs& a, cudaStream_t st) {
             S = s;
             break;
         }
-    return launch_clustered(fused_mt_kernel<DT, TMAX, IN, EP, STAGES>, S, rows, dyn, b, st);
+    return launch_clustered(fused_mt_kernel<DT, TMAX, IN, EP, STAGES, CAPM, BPS>, S, rows, dyn, b, st);
 }
 
+// One block per SM (the inputs of several tokens and the tensor-core buffers fill its shared
+// memory): 6 pipeline stages, 3 where 8 tokens of a wide model leave less.  (Two blocks per SM
+// with the buffers inside the histogram's 64 KB -- 512 staged entries per pass, 3 stages, twice
+// as many blocks to share the per-token selections -- measured slower: 295 instead of 255 us per
+// 13B layer at 4 tokens.)
 template <int DT, int TMAX, int IN, int EP>
 static afx_status launch_fused_mt(const FusedArgs& a, cudaStream_t st) {
     if (static_cast<uint64_t>(a.K) * static_cast<uint64_t>(a.ldw >> 3) > 0x100000000ull) return AFX_ERR_CAPACITY;
-    if (fused_dyn_smem(IN, a.K, a.T, sizeof(MtSmem<FusedMtCap<TMAX>::value, kFusedMtStages>)) <= kMaxDynSmem)
-        return launch_fused_mt_st<DT, TMAX, IN, EP, kFusedMtStages>(a, st);
-    if (fused_dyn_smem(IN, a.K, a.T, sizeof(MtSmem<FusedMtCap<TMAX>::value, kFusedMtStagesSmall>)) <= kMaxDynSmem)
-        return launch_fused_mt_st<DT, TMAX, IN, EP, kFusedMtStagesSmall>(a, st);
+    constexpr int kCap1 = FusedMtCap<TMAX>::value;
+    if (fused_dyn_smem(IN, a.K, a.T, sizeof(MtSmem<kCap1, kFusedMtStages>)) <= kMaxDynSmem)
+        return launch_fused_mt_st<DT, TMAX, IN, EP, kFusedMtStages, kCap1, 1>(a, st);
+    if (fused_dyn_smem(IN, a.K, a.T, sizeof(MtSmem<kCap1, kFusedMtStagesSmall>)) <= kMaxDynSmem)
+        return launch_fused_mt_st<DT, TMAX, IN, EP, kFusedMtStagesSmall, kCap1, 1>(a, st);
     return AFX_ERR_CAPACITY;
 }
 
