@@ -32,7 +32,7 @@ constexpr int kFusedMtStages = 6, kFusedMtStagesSmall = 3;  // pipeline stages o
 constexpr size_t kMaxDynSmem = 227 * 1024;
 template <int TMAX>
 struct FusedMtCap {
-    static constexpr int value = TMAX <= 4 ? 2048 : 1024;
+    static constexpr int value = TMAX <= 4 ? 4096 : 1024;
 };
 // CAPM staged entries per pass, STAGES pipeline stages, BPS blocks per SM.
 template <int DT, int TMAX, int IN, int EP, int STAGES, int CAPM, int BPS>
