@@ -116,6 +116,28 @@ def test_chain_without_synchronisation_gives_the_same_bits(NL, depth, xl_mode, h
     m.close()
 
 
+@pytest.mark.parametrize("T,depth", [(4, 1), (8, 0), (2, 3)])
+def test_chain_without_synchronisation_with_several_tokens_per_step(T, depth):
+    """The same with several tokens per step: the blocks of a cluster exchange the per-token
+    sets through distributed shared memory and the streaming stage runs on the tensor cores;
+    launches that overlap must still give the bits of the synchronised run."""
+    dt, NL, heads, kvh, mlp, max_seq, pos, n_tokens = "bf16", 4, 2, 1, 512, 40, 20, 4
+    xl_mode = afx.XL_BOOKKEEP if depth else afx.XL_OFF
+    cfg, k, layers, lws, caches, m = small_model(49, NL, dt, heads, kvh, mlp, T, max_seq, pos, depth, xl_mode)
+    h0 = synth.hidden_state(49, 5, T, cfg.hidden, scale=4.0, scales_stream=6)
+    ref = run_tokens(m, h0, n_tokens, NL, pos, sync=True)
+    for attempt in range(4):
+        got = run_tokens(m, h0, n_tokens, NL, pos, sync=False)
+        assert np.array_equal(got["h"].view(np.uint32), ref["h"].view(np.uint32)), attempt
+        assert np.array_equal(got["stats"], ref["stats"]), attempt
+        for op in range(4):
+            n_idx = ref["stats"][NL - 1][op][0]
+            assert np.array_equal(got["idx"][op][:n_idx], ref["idx"][op][:n_idx])
+        for l in range(NL):
+            assert np.array_equal(got["kc"][l], ref["kc"][l]) and np.array_equal(got["vc"][l], ref["vc"][l])
+    m.close()
+
+
 def test_one_layer_several_tokens_each_against_the_oracle():
     """One layer stepped over successive positions: every token's stages against the oracle on
     the cache the GPU has built so far (rows written by earlier tokens are read back)."""
