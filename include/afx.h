@@ -112,7 +112,10 @@ afx_status afx_diff_active(const int32_t* idxA, const int32_t* cntA, const uint3
  *
  * with col(c) = idx[c], or slot[c] when `slot` is given (the columns then live in a cache
  * whose slot list afx_cache_fetch produced).  Products are exact in fp32; sums are fp32 in
- * a fixed order (same inputs on the same device give the same bits).
+ * a fixed order (same inputs on the same device give the same bits).  One token is multiplied
+ * on the fp32 pipe; with 2..8 tokens the active rows are gathered into shared memory and
+ * multiplied on the tensor cores (16-bit inputs, fp32 accumulation): the order of the sums, and
+ * with it the last bits of y, differ between the two, the rules above hold for both.
  *
  *   Wt        DEVICE, channel-contiguous weights (see the conventions above).
  *   x         DEVICE, [T][K] 16-bit floats; every token uses the whole list.
