@@ -47,6 +47,8 @@ struct FusedArgs {
     int32_t* kth_slot;
     // ---- the same for several tokens (T > 1; may be NULL): T consecutive slots, one per token ----
     int32_t* kth_multi;
+    // ---- set by the launcher (several-token operators): column tiles per cluster, 0 or 1 = one ----
+    int tiles_per_cluster;
     // ---- set by the launcher: 1 if the grid has one more cluster than column tiles; its block 0
     // repeats input stage and selection only to write the side outputs, off the path of the
     // clusters that stream (its other blocks leave at once) ----
@@ -90,10 +92,15 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int warp = tid >> 5;
-    const int S = gridDim.x, s = blockIdx.x;
+    // CS blocks form a cluster; S of them split the active list of one column tile.  CS == S
+    // except for several-token operators with few tiles: there a cluster covers CS / S adjacent
+    // tiles, so that more blocks share the per-token selections (a.tiles_per_cluster).
+    const int CS = gridDim.x, cs = blockIdx.x;
+    const int tpc = (WMT > 0 && a.tiles_per_cluster > 1) ? a.tiles_per_cluster : 1;
+    const int S = tpc > 1 ? CS / tpc : CS, s = tpc > 1 ? cs % S : cs;
     const int T = a.T, K = a.K;
     const bool side = a.side_cluster != 0 && blockIdx.y == gridDim.y - 1;  // the cluster without a tile
-    int tile = blockIdx.y, grp = 0;
+    int tile = tpc > 1 ? blockIdx.y * tpc + cs / S : blockIdx.y, grp = 0;
     if (GRP && a.groups > 1) {  // (never together with a side cluster)
         const int per = gridDim.y / a.groups;
         grp = tile / per;
@@ -249,10 +256,10 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
     uint32_t* xchg = kXchgFits ? reinterpret_cast<uint32_t*>(work + kXchgOffset) : nullptr;
     bool first_staged = false;
     // Several tokens: the blocks of a cluster share the work -- block s decides the sets of the
-    // tokens t with t % S == s and writes their flags into every block's table of per-token
+    // tokens t with t % CS == cs and writes their flags into every block's table of per-token
     // bitmaps (distributed shared memory); after one cluster barrier every thread reads the
     // union for its own chunks.  (The side cluster works alone and decides every token.)
-    const bool share = TMAX > 1 && T > 1 && own && !side && S > 1;
+    const bool share = TMAX > 1 && T > 1 && own && !side && CS > 1;
     uint8_t* const ftab = dyn + fused_input_smem(IN, K, T);
     const size_t fstride = fused_flag_smem(K);
     if (own) {
@@ -260,7 +267,7 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
         if (share) cluster_wait();  // pairs with the cluster_arrive() at kernel start: the peers are running
         bool first = true;
         for (int t = 0; t < T; ++t) {
-            if (share && t % S != s) continue;
+            if (share && t % CS != cs) continue;
             const uint16_t* xt = xs + (IN == IN_NORM ? static_cast<size_t>(t) * Kp : 0);
             if (IN == IN_X) {
                 if (!first) __syncthreads();  // the previous token's keys are still being read
@@ -290,7 +297,7 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
                 if (share) {
                     int q_lo, q_hi;
                     thread_chunk_range(K, q_lo, q_hi);
-                    for (int q = 0; q < S; ++q) {
+                    for (int q = 0; q < CS; ++q) {
                         uint8_t* dst = cg::this_cluster().map_shared_rank(ftab + static_cast<size_t>(t) * fstride, q);
                         for (int c = q_lo; c < q_hi; ++c) dst[c] = static_cast<uint8_t>(ft >> (8 * (c - q_lo)));
                     }
@@ -365,8 +372,10 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
         constexpr int kMtCap = CAP;
         float c4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
         const uint4* wtile16 = reinterpret_cast<const uint4*>(Wt + static_cast<size_t>(tile) * kMtTile);
-        const int n_chunks = min(kMtTile, a.N - tile * kMtTile) >> 3;
-        for (int c0 = c_lo; c0 < c_hi; c0 += kMtCap) {
+        const int n_chunks = max(0, min(kMtTile, a.N - tile * kMtTile)) >> 3;
+        // (the last cluster of a grid with several tiles per cluster may hold a block without a
+        // tile: it only shares the selections and meets the barriers)
+        for (int c0 = c_lo; n_chunks > 0 && c0 < c_hi; c0 += kMtCap) {
             const int staged = min(kMtCap, c_hi - c0);
             __syncthreads();  // the work area is free: the histogram / the previous pass has been read
             if (own) {
@@ -396,7 +405,7 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
         }
         EpilogueArgs ep = a.ep;
         if (!share) cluster_wait();  // pairs with the cluster_arrive() at kernel start
-        mt_finish<DT>(c4, mt, T, tile, a.N, EP, ep);
+        mt_finish<DT>(c4, mt, T, tile, a.N, EP, ep, S, s, cs - s);
         return;
     }
     for (int c0 = c_lo; c0 < c_hi; c0 += CAP) {

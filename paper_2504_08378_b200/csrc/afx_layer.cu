@@ -163,16 +163,28 @@ static afx_status launch_fused_mt_st(const FusedArgs& a, cudaStream_t st) {
                       a.kth_multi != nullptr)
                          ? 1 : 0;
     const int tiles = (a.N + kMtTile - 1) / kMtTile;
-    const int rows = tiles + b.side_cluster;
-    if (rows > 65535) return AFX_ERR_CAPACITY;
+    if (tiles + b.side_cluster > 65535) return AFX_ERR_CAPACITY;
     const int margin = (tiles + 15) / 16 < 2 ? 2 : (tiles + 15) / 16;
     int S = 1;
     for (int s = kMaxCluster; s > 1; --s)
-        if (max_active_clusters(kern, s, dyn) >= rows + margin) {
+        if (max_active_clusters(kern, s, dyn) >= tiles + b.side_cluster + margin) {
             S = s;
             break;
         }
-    return launch_clustered(fused_mt_kernel<DT, TMAX, IN, EP, STAGES, CAPM, BPS>, S, rows, dyn, b, st);
+    // Few tiles leave the clusters smaller than the number of tokens: let a cluster cover several
+    // adjacent tiles, so that its blocks share the per-token selections (own selection only).
+    int tpc = 1;
+    if (a.idx_in == nullptr)
+        for (int t2 = 8; t2 > 1; t2 >>= 1) {
+            const int cs = S * t2, rows2 = (tiles + t2 - 1) / t2 + b.side_cluster;
+            if (cs <= kMaxCluster && cs <= 2 * a.T && max_active_clusters(kern, cs, dyn) >= rows2 + (margin + t2 - 1) / t2) {
+                tpc = t2;
+                break;
+            }
+        }
+    b.tiles_per_cluster = tpc;
+    const int rows = (tiles + tpc - 1) / tpc + b.side_cluster;
+    return launch_clustered(fused_mt_kernel<DT, TMAX, IN, EP, STAGES, CAPM, BPS>, S * tpc, rows, dyn, b, st);
 }
 
 // One block per SM (the inputs of several tokens and the tensor-core buffers fill its shared

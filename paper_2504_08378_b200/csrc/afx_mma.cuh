@@ -148,13 +148,17 @@ __device__ __forceinline__ void mt_pad_inputs(SMT* sm, int T, int staged) {
 // The cluster's partial sums meet in rank order, then the epilogue (EP_STORE / EP_ACCUM /
 // EP_SILU as in gemv_finish_tile).  Every thread of every block of the cluster calls it; no
 // cluster barrier arrival may be pending.
+// S blocks of the cluster, ranks base .. base + S - 1, worked on this tile; the caller is the
+// rank-th of them (S < 0: the whole cluster).
 template <int DT, class SMT>
 __device__ __forceinline__ void mt_finish(const float (&c)[4], SMT* sm, int T, int tile, int N, int ep_kind,
-                                          const EpilogueArgs& ep) {
+                                          const EpilogueArgs& ep, int S = -1, int rank = 0, int base = 0) {
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
-    const int S = static_cast<int>(cluster.num_blocks());
-    const int rank = static_cast<int>(cluster.block_rank());
+    if (S < 0) {
+        S = static_cast<int>(cluster.num_blocks());
+        rank = static_cast<int>(cluster.block_rank());
+    }
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     __syncthreads();  // the last stage has been multiplied by everybody
     float* part = reinterpret_cast<float*>(sm->w[0]);  // [8 tokens][kMtPartStride]
@@ -176,7 +180,7 @@ __device__ __forceinline__ void mt_finish(const float (&c)[4], SMT* sm, int T, i
             if (2 * m < N) {
                 float g = 0.0f, u = 0.0f;
                 for (int q = 0; q < S; ++q) {
-                    const float* pq = cluster.map_shared_rank(part, q) + t * kMtPartStride;
+                    const float* pq = cluster.map_shared_rank(part, base + q) + t * kMtPartStride;
                     g += pq[og];
                     u += pq[og + 8];
                 }
@@ -190,7 +194,7 @@ __device__ __forceinline__ void mt_finish(const float (&c)[4], SMT* sm, int T, i
             const int out = tile * kMtTile + o;
             if (out < N) {
                 float s = 0.0f;
-                for (int q = 0; q < S; ++q) s += cluster.map_shared_rank(part, q)[t * kMtPartStride + o];
+                for (int q = 0; q < S; ++q) s += cluster.map_shared_rank(part, base + q)[t * kMtPartStride + o];
                 s *= out_scale;
                 float* p = ep.y + static_cast<size_t>(t) * N + out;
                 *p = ep_kind == EP_ACCUM ? *p + s : s;
