@@ -14,6 +14,8 @@ namespace afx {
 
 enum { IN_X = 0, IN_NORM = 1 };
 
+constexpr int kFusedMtRows = 64;  // channels per pipeline stage of the several-token operator
+
 struct FusedArgs {
     const uint16_t* Wt;
     // mixture of experts: if wt_table is given, the weights are wt_table[*wt_sel] (both DEVICE;
@@ -367,7 +369,7 @@ __device__ __forceinline__ void fused_op_block(const FusedArgs& a, unsigned char
 
     const int n_mine = __popcll(fl);
     if (WMT) {
-        using MtT = MtSmem<CAP, (WMT > 0 ? WMT : 2)>;
+        using MtT = MtSmem<CAP, (WMT > 0 ? WMT : 2), kFusedMtRows>;
         MtT* mt = reinterpret_cast<MtT*>(work);
         constexpr int kMtCap = CAP;
         float c4[4] = {0.0f, 0.0f, 0.0f, 0.0f};

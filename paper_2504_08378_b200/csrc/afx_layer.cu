@@ -28,11 +28,11 @@ fused_op_kernel(FusedArgs a) {
 
 // The operator for several tokens per step: the streaming stage runs on the tensor cores.  The
 // block is alone on its SM: staged entries per pass as many as the inputs of TMAX tokens leave room for.
-constexpr int kFusedMtStages = 6, kFusedMtStagesSmall = 3;  // pipeline stages of the several-token operator
+constexpr int kFusedMtStages = 3, kFusedMtStagesSmall = 2;  // pipeline stages of the several-token operator
 constexpr size_t kMaxDynSmem = 227 * 1024;
 template <int TMAX>
 struct FusedMtCap {
-    static constexpr int value = TMAX <= 4 ? 4096 : 1024;
+    static constexpr int value = TMAX <= 4 ? 4096 : 1024;  // (multiples of kFusedMtRows)
 };
 // CAPM staged entries per pass, STAGES pipeline stages, BPS blocks per SM.
 template <int DT, int TMAX, int IN, int EP, int STAGES, int CAPM, int BPS>
@@ -156,7 +156,7 @@ static afx_status launch_fused_q4(int dtype, const FusedArgs& a, cudaStream_t st
 template <int DT, int TMAX, int IN, int EP, int STAGES, int CAPM, int BPS>
 static afx_status launch_fused_mt_st(const FusedArgs& a, cudaStream_t st) {
     const void* kern = reinterpret_cast<const void*>(fused_mt_kernel<DT, TMAX, IN, EP, STAGES, CAPM, BPS>);
-    const size_t dyn = fused_dyn_smem(IN, a.K, a.T, sizeof(MtSmem<CAPM, STAGES>));
+    const size_t dyn = fused_dyn_smem(IN, a.K, a.T, sizeof(MtSmem<CAPM, STAGES, kFusedMtRows>));
     FusedArgs b = a;
     b.side_cluster = (a.idx_out != nullptr || a.count_out != nullptr || a.bitmap_out != nullptr ||
                       a.xnorm_out != nullptr || a.bitmap_pred != nullptr || a.kth_slot != nullptr ||
@@ -196,9 +196,9 @@ template <int DT, int TMAX, int IN, int EP>
 static afx_status launch_fused_mt(const FusedArgs& a, cudaStream_t st) {
     if (static_cast<uint64_t>(a.K) * static_cast<uint64_t>(a.ldw >> 3) > 0x100000000ull) return AFX_ERR_CAPACITY;
     constexpr int kCap1 = FusedMtCap<TMAX>::value;
-    if (fused_dyn_smem(IN, a.K, a.T, sizeof(MtSmem<kCap1, kFusedMtStages>)) <= kMaxDynSmem)
+    if (fused_dyn_smem(IN, a.K, a.T, sizeof(MtSmem<kCap1, kFusedMtStages, kFusedMtRows>)) <= kMaxDynSmem)
         return launch_fused_mt_st<DT, TMAX, IN, EP, kFusedMtStages, kCap1, 1>(a, st);
-    if (fused_dyn_smem(IN, a.K, a.T, sizeof(MtSmem<kCap1, kFusedMtStagesSmall>)) <= kMaxDynSmem)
+    if (fused_dyn_smem(IN, a.K, a.T, sizeof(MtSmem<kCap1, kFusedMtStagesSmall, kFusedMtRows>)) <= kMaxDynSmem)
         return launch_fused_mt_st<DT, TMAX, IN, EP, kFusedMtStagesSmall, kCap1, 1>(a, st);
     return AFX_ERR_CAPACITY;
 }
@@ -377,8 +377,8 @@ extern "C" afx_status afx_state_create(const afx_model* model, int T, void* blob
     // the widest input stage must fit one block's shared memory
     const size_t dyn_max = afx::fused_dyn_smem(
         afx::IN_NORM, model->d.hidden, T,
-        T > 4 ? sizeof(afx::MtSmem<afx::FusedMtCap<8>::value, afx::kFusedMtStagesSmall>)
-              : (T > 1 ? sizeof(afx::MtSmem<afx::FusedMtCap<4>::value, afx::kFusedMtStagesSmall>) : 0));
+        T > 4 ? sizeof(afx::MtSmem<afx::FusedMtCap<8>::value, afx::kFusedMtStagesSmall, afx::kFusedMtRows>)
+              : (T > 1 ? sizeof(afx::MtSmem<afx::FusedMtCap<4>::value, afx::kFusedMtStagesSmall, afx::kFusedMtRows>) : 0));
     if (dyn_max > afx::kMaxDynSmem || model->d.mlp > afx::kSelectFastMaxK ||
         model->d.n_heads * model->d.head_dim > afx::kSelectFastMaxK) {
         delete s;

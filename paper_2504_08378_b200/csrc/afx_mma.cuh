@@ -23,23 +23,25 @@ namespace afx {
 
 constexpr int kMtTokens = 8;                      // token rows of the B operand (rows >= T hold zeros)
 constexpr int kMtTile = 256;                      // outputs per cluster
-constexpr int kMtStageRows = 32;                  // channels per pipeline stage
 constexpr int kMtRowBytes = kMtTile * 2 + 16;     // a staged channel row (+16 bytes: ldmatrix rows fall into different banks)
-constexpr int kMtStageBytes = kMtStageRows * kMtRowBytes;
 constexpr int kMtPartStride = kMtTile + 4;        // floats per token row of the partial sums
 
-// CAPM = staged list entries per pass (a multiple of kMtStageRows): every pass fills and drains
+// CAPM = staged list entries per pass (a multiple of ROWS): every pass fills and drains
 // the pipeline once, so a block that is alone on its SM takes a large one.
 // STAGES = pipeline stages (STAGES - 1 of them in flight while one is multiplied).
-template <int CAPM, int STAGES>
+// ROWS = channels per stage (a multiple of 16).
+template <int CAPM, int STAGES, int ROWS = 32>
 struct MtSmem {
     static constexpr int kCap = CAPM;
     static constexpr int kStages = STAGES;
+    static constexpr int kRows = ROWS;
+    static constexpr int kStageBytes = ROWS * kMtRowBytes;
+    static_assert(ROWS % 16 == 0 && CAPM % ROWS == 0 && kMtTokens * kMtPartStride * 4 <= ROWS * kMtRowBytes,
+                  "stage shape (the partial sums reuse the first stage buffer)");
     uint32_t col[CAPM];                                // row offset of a staged channel in 16-byte units
     __align__(16) uint16_t xb[kMtTokens][CAPM + 8];    // the tokens' inputs at the staged channels (+16 bytes per row: no bank conflicts)
-    __align__(16) unsigned char w[STAGES][kMtStageBytes];
+    __align__(16) unsigned char w[STAGES][ROWS * kMtRowBytes];
 };
-static_assert(kMtTokens * kMtPartStride * 4 <= kMtStageBytes, "partial sums reuse the first stage buffer");
 
 __device__ __forceinline__ uint32_t mt_smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -67,7 +69,7 @@ __device__ __forceinline__ void mt_mma(float (&c)[4], const uint32_t (&a)[4], ui
 }
 
 // One pass over the staged channels [0, staged) (sm->col, sm->xb filled, zero x behind `staged`
-// up to the end of the last stage, a block barrier since): kStages - 1 stages of kMtStageRows
+// up to the end of the last stage, a block barrier since): kStages - 1 stages of kRows
 // channels in flight while one is multiplied.  wtile16 = the weights at this tile's first output;
 // n_chunks = valid 16-byte pieces per row of the tile (pieces beyond the operator's last output
 // and rows at or beyond `staged` are filled with zeros).  Every thread of the block calls it; on
@@ -77,6 +79,8 @@ __device__ __forceinline__ void mt_mma(float (&c)[4], const uint32_t (&a)[4], ui
 template <int DT, class SMT>
 __device__ __forceinline__ void mt_stream_pass(const uint4* wtile16, SMT* sm, int staged, int n_chunks, float (&c)[4]) {
     constexpr int kSt = SMT::kStages;
+    constexpr int kMtStageRows = SMT::kRows;
+    constexpr int kMtStageBytes = SMT::kStageBytes;
     constexpr int kChunks = kMtTile / 8;                       // 16-byte pieces per row
     constexpr int kSweep = kGemvThreads / kChunks;             // rows the block copies at once
     static_assert(kChunks == 32 && kMtStageRows % kSweep == 0, "copy pattern");
@@ -138,6 +142,7 @@ __device__ __forceinline__ void mt_stream_pass(const uint4* wtile16, SMT* sm, in
 // token rows that hold no token: whatever the multiply reads there must be 0 (no barrier).
 template <class SMT>
 __device__ __forceinline__ void mt_pad_inputs(SMT* sm, int T, int staged) {
+    constexpr int kMtStageRows = SMT::kRows;
     const int padded = (staged + kMtStageRows - 1) / kMtStageRows * kMtStageRows;
     for (int i = staged + threadIdx.x; i < padded; i += kGemvThreads)
         for (int t = 0; t < T; ++t) sm->xb[t][i] = 0;
