@@ -188,7 +188,7 @@ static afx_status launch_fused_mt_st(const FusedArgs& a, cudaStream_t st) {
 }
 
 // One block per SM (the inputs of several tokens and the tensor-core buffers fill its shared
-// memory): 6 pipeline stages, 3 where 8 tokens of a wide model leave less.  (Two blocks per SM
+// memory): 3 pipeline stages of 64 channels, 2 where 8 tokens of a wide model leave less.  (Two blocks per SM
 // with the buffers inside the histogram's 64 KB -- 512 staged entries per pass, 3 stages, twice
 // as many blocks to share the per-token selections -- measured slower: 295 instead of 255 us per
 // 13B layer at 4 tokens.)
