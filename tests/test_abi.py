@@ -107,3 +107,43 @@ def test_diff_rejects_bad_arguments_on_the_host():
     assert _status(afx.afx_diff_active, None, FAKE, FAKE, 8, FAKE, FAKE, FAKE) == 1
     assert _status(afx.afx_diff_active, FAKE, FAKE, FAKE, 0, FAKE, FAKE, FAKE) == 1
     assert _status(afx.afx_diff_active, FAKE + 2, FAKE, FAKE, 8, FAKE, FAKE, FAKE) == 2
+
+
+def test_binding_structs_have_the_headers_layout(tmp_path):
+    """Every ctypes structure of the binding against the C compiler's view of include/afx.h:
+    same size, same offset of every field (the header is plain C: gcc compiles it)."""
+    pairs = {"afx_model_desc": afx.ModelDesc, "afx_layer_desc": afx.LayerDesc, "afx_cache_desc": afx.CacheDesc,
+             "afx_cache_stats": afx.CacheStats, "afx_swap_desc": afx.SwapDesc, "afx_swap_stats": afx.SwapStats,
+             "afx_cost_params": afx.CostParams, "afx_cost": afx.Cost, "afx_cost_search_in": afx.CostSearchIn,
+             "afx_cost_choice": afx.CostChoice, "afx_moe_desc": afx.MoeDesc, "afx_hosted_ops": afx.HostedOps,
+             "afx_q4_layer": afx.Q4Layer}
+    hdr = open(os.path.join(ROOT, "include", "afx.h")).read()
+    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+    lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "afx.h"', "int main(void) {"]
+    fields = {}
+    for cname in pairs:
+        body = re.search(r"typedef struct \{([^}]*)\}\s*" + cname + r"\s*;", hdr).group(1)
+        names = []
+        for decl in body.split(";"):
+            decl = decl.strip()
+            if decl:
+                for part in decl.split(","):
+                    names.append(re.search(r"([A-Za-z_][A-Za-z0-9_]*)\s*(\[[^\]]*\])?\s*$", part.strip()).group(1))
+        fields[cname] = names
+        lines.append(f'  printf("{cname} %zu", sizeof({cname}));')
+        for n in names:
+            lines.append(f'  printf(" %zu", offsetof({cname}, {n}));')
+        lines.append('  printf("\\n");')
+    lines += ["  return 0;", "}"]
+    src = tmp_path / "layout.c"
+    src.write_text("\n".join(lines))
+    exe = tmp_path / "layout"
+    subprocess.check_call(["gcc", "-I", os.path.join(ROOT, "include"), "-o", str(exe), str(src)])
+    out = subprocess.check_output([str(exe)], text=True)
+    for ln in out.splitlines():
+        cname, size, *offs = ln.split()
+        cls = pairs[cname]
+        assert ctypes.sizeof(cls) == int(size), cname
+        py_names = [f[0] for f in cls._fields_]
+        assert py_names == fields[cname], (cname, py_names, fields[cname])
+        assert [getattr(cls, n).offset for n in py_names] == [int(o) for o in offs], cname
