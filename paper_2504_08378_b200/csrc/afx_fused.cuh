@@ -5,6 +5,9 @@
 // selection launch, no count/index round trips through global memory.
 #pragma once
 
+// (the several-token instantiations leave fused_op_block before its one-token streaming loop)
+#pragma nv_diag_suppress 128
+
 #include "afx_gemv.cuh"
 #include "afx_mma.cuh"
 #include "afx_q4.cuh"
